@@ -1,0 +1,187 @@
+/*
+ * lsp.h -- C ABI of the B200 (sm_100a) Longest-Stable-Prefix decode library.
+ *
+ * The library runs the per-step hot path of the LSP scheduler for diffusion language models:
+ * one bidirectional denoiser pass over [pending block | masked suffix] with the committed prefix
+ * served from a contiguous KV cache (Algorithm 1 line 4), the fused LM-head + confidence
+ * reduction (Eq. 1 and the softmax max-probability; line 5), the longest-stable-run scan with
+ * adaptive threshold (Eq. 2), delimiter snap and fallback (lines 6-8), and the atomic commit with
+ * the contiguous KV append (lines 9-10).
+ *
+ * Conventions
+ *  - Every function returns 0 on success or a negative LSP_ERR_* code; lsp_last_error() gives text.
+ *  - "device" pointers are CUDA global memory of the current device; "host" pointers are ordinary
+ *    host memory.  The library never allocates device memory: weights, KV cache, workspace, token
+ *    buffer and the stream belong to the caller and are borrowed until lsp_destroy().
+ *  - Work is enqueued on the stream given to lsp_init().  A call that returns host-visible results
+ *    synchronises that stream (only); the others return as soon as the work is enqueued.
+ *  - Element type T is float (dtype 0) or bfloat16 (dtype 1).  bf16 GEMMs run on tcgen05 tensor
+ *    cores with fp32 accumulation; fp32 models run on CUDA cores.
+ *  - All linear weights are row-major [out_features, in_features] (K-major operands).
+ */
+#ifndef LSP_H_
+#define LSP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LSP_OK 0
+#define LSP_ERR_ARG (-1)            /* NULL pointer, negative size, bad enum value */
+#define LSP_ERR_SHAPE (-2)          /* model shape not supported (see lsp_init) */
+#define LSP_ERR_WORKSPACE (-3)      /* workspace smaller than lsp_workspace_bytes() */
+#define LSP_ERR_STATE (-4)          /* call out of order, L out of range, decode already finished */
+#define LSP_ERR_CUDA (-5)           /* a CUDA runtime/driver call failed */
+#define LSP_ERR_DEVICE_TIMEOUT (-6) /* a bounded device-side wait expired; results of the step are invalid */
+
+/* flags in lsp_step_rec.flags */
+#define LSP_FLAG_SNAPPED 1u
+#define LSP_FLAG_FALLBACK 2u
+#define LSP_FLAG_RANGE_UNACHIEVABLE 4u
+#define LSP_FLAG_RUN_TO_END 8u
+#define LSP_FLAG_NEAR_THRESHOLD 16u
+#define LSP_FLAG_NEAR_TIE 32u
+
+typedef struct lsp_ctx lsp_ctx;
+
+/* Transformer shape (the paper treats p_theta as a black box; the shape is the benchmark's):
+ * pre-norm blocks, RMSNorm, rotary positions with rotate-half pairing (i, i + head_dim/2),
+ * non-causal attention (n_heads query heads, n_kv_heads key/value heads), SwiGLU FFN, no biases,
+ * untied head.  Requirements: head_dim in {64, 128}; d_model, d_ffn, n_heads*head_dim multiples
+ * of 64; n_heads % n_kv_heads == 0. */
+typedef struct {
+  int n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rms_eps, rope_theta;
+  int dtype;   /* 0 = fp32, 1 = bf16 */
+  int mask_id; /* id of the [MASK] token */
+} lsp_model_cfg;
+
+/* Scheduler policy (Sec. 3.2; Algorithm 1 inputs). */
+typedef struct {
+  int score;       /* 0 = softmax max-probability, 1 = logit margin delta_i (Eq. 1) */
+  int mode;        /* 0 = fixed threshold tau, 1 = adaptive tau with L' in [alpha N, beta N] (Eq. 2),
+                      2 = commit exactly fixed_k tokens per step (ablation policy, no snapping) */
+  float tau, alpha, beta;
+  int l_min;       /* L_min >= 1 */
+  int snap_window; /* W >= 0; negative = unbounded look-back */
+  int fixed_k;
+  const uint8_t* delim_bitmap; /* device, (vocab+7)/8 bytes, bit (v & 7) of byte v >> 3; NULL = empty set D */
+  int exclude_mask_logit;      /* 1: the mask_id column takes no part in argmax / margin / probability */
+  float flag_tol;              /* tolerance of the NEAR_THRESHOLD / NEAR_TIE flags; 0 disables them */
+} lsp_sched_cfg;
+
+/* Device pointers to the weights, all element type T.  Per-layer arrays are HOST arrays of
+ * n_layers device pointers.  w_qkv rows: n_heads*head_dim query rows, then n_kv_heads*head_dim key
+ * rows, then n_kv_heads*head_dim value rows. */
+typedef struct {
+  const void* embed;       /* [vocab, d_model] */
+  const void* final_norm;  /* [d_model] */
+  const void* w_head;      /* [vocab, d_model] */
+  const void* const* attn_norm; /* [d_model] */
+  const void* const* w_qkv;     /* [(n_heads + 2 n_kv_heads) head_dim, d_model] */
+  const void* const* w_o;       /* [d_model, n_heads head_dim] */
+  const void* const* ffn_norm;  /* [d_model] */
+  const void* const* w_gate;    /* [d_ffn, d_model] */
+  const void* const* w_up;      /* [d_ffn, d_model] */
+  const void* const* w_down;    /* [d_model, d_ffn] */
+} lsp_weights;
+
+/* One record per sequence and step. */
+typedef struct {
+  int step;      /* step index k */
+  int n_before;  /* N_k, active positions before the commit */
+  int rows;      /* query rows this sequence contributed to the pass (pending block + N_k) */
+  int l_run;     /* L' */
+  int l_commit;  /* L */
+  float tau_used;
+  unsigned flags;
+  float ms;      /* device time of the whole step (same value for every sequence of the batch) */
+} lsp_step_rec;
+
+/* Bytes of workspace lsp_init() needs for up to max_batch sequences of up to max_len positions
+ * (prompt + generation).  Includes the staging buffer that holds one pass's K/V for all layers. */
+size_t lsp_workspace_bytes(const lsp_model_cfg* model, int max_batch, int max_len);
+
+/* Bytes of the contiguous prefix KV cache: [n_layers][2][max_batch][max_len][n_kv_heads*head_dim] T. */
+size_t lsp_kv_cache_bytes(const lsp_model_cfg* model, int max_batch, int max_len);
+
+/* Creates a context.  kv_cache and workspace are device buffers of at least the sizes above, 256-byte
+ * aligned; cuda_stream is a cudaStream_t (NULL = default stream).  The first call builds the rotary
+ * table on the device and may JIT nothing; it does not allocate device memory. */
+int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sched, const lsp_weights* weights,
+             void* kv_cache, void* workspace, size_t workspace_bytes, int max_batch, int max_len,
+             void* cuda_stream);
+
+/* Replaces the scheduler policy (allowed between steps). */
+int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
+
+/* Options: key 0 = GEMM implementation for bf16 (0 = CUDA-core reference kernels, 1 = tcgen05,
+ * default 1); key 1 = attention implementation for bf16 (0 = CUDA-core, 1 = tensor-core). */
+int lsp_set_option(lsp_ctx* ctx, int key, int value);
+
+/* Algorithm 1 line 2: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32
+ * [batch, token_stride], caller-owned, prompt ids already at [0, prompt_len[b]); the library writes
+ * mask_id over [prompt_len[b], prompt_len[b]+gen_len[b]) and later the committed ids.  prompt_len,
+ * gen_len: host [batch].  prompt_len[b] >= 1, gen_len[b] >= 1, sum <= max_len, <= token_stride. */
+int lsp_begin(lsp_ctx* ctx, int32_t* tokens, int token_stride, const int32_t* prompt_len,
+              const int32_t* gen_len, int batch);
+
+/* Algorithm 1 lines 4-8 for every unfinished sequence: the pass, the scores, the scan; proposes L
+ * and changes no committed state.  rec: host [batch] or NULL.  Synchronises the stream. */
+int lsp_denoise_step(lsp_ctx* ctx, lsp_step_rec* rec);
+
+/* Algorithm 1 lines 9-10: writes yhat_{1:L} into the token buffer, appends the pending block's K/V
+ * (computed by the last pass) to the cache as one contiguous copy per layer, and makes the new
+ * block pending.  L_override: host [batch] (entries of finished sequences ignored) or NULL to use the
+ * proposed lengths.  Needs a preceding lsp_denoise_step; 1 <= L <= N_b else LSP_ERR_STATE and nothing
+ * changes.  Asynchronous. */
+int lsp_commit(lsp_ctx* ctx, const int32_t* L_override);
+
+/* Algorithm 1 lines 3-11: step + commit until every sequence is fully committed.  recs: host
+ * [max_recs] records in (step, sequence) order, or NULL; n_steps: number of denoiser passes. */
+int lsp_generate(lsp_ctx* ctx, lsp_step_rec* recs, int max_recs, int* n_steps);
+
+/* Number of still-active positions per sequence (host [batch]); returns the count of unfinished sequences
+ * through *n_unfinished. */
+int lsp_active(lsp_ctx* ctx, int32_t* n_active, int* n_unfinished);
+
+/* Per-position outputs of the last step / last lsp_head_scan, copied to host arrays of
+ * lsp_score_rows() entries (sequence-major, active positions in order).  Any pointer may be NULL. */
+int lsp_score_rows(lsp_ctx* ctx);
+int lsp_get_scores(lsp_ctx* ctx, int32_t* yhat, float* pmax, float* margin);
+
+/* The fused LM-head + confidence reduction and the scan alone (Eq. 1, Eq. 2, snapping), on hidden
+ * states the caller provides: hidden device [rows, d_model] T (used as given: no normalisation),
+ * seq_offsets host [batch+1] ascending with seq_offsets[batch] = rows <= max_batch*max_len.
+ * Outputs host [batch] each (may be NULL).  Full-vocabulary logits are never written to memory.
+ * Synchronises the stream. */
+int lsp_head_scan(lsp_ctx* ctx, const void* hidden, const int32_t* seq_offsets, int batch, int32_t* l_run,
+                  int32_t* l_commit, uint32_t* flags, float* tau_used);
+
+/* The scan alone on caller-provided device arrays score[rows] (fp32), yhat[rows]; margin may be NULL.
+ * Same outputs as lsp_head_scan. */
+int lsp_scan(lsp_ctx* ctx, const float* score, const int32_t* yhat, const float* margin,
+             const int32_t* seq_offsets, int batch, int32_t* l_run, int32_t* l_commit, uint32_t* flags,
+             float* tau_used);
+
+/* Kernel-level entry points used for parity checks at full shapes (device pointers, element type T
+ * of the context).  op: 0 = out[M,N] = A W^T; 1 = out[M,N] += A W^T (residual update);
+ * 2 = out[M,N] = silu(A W^T) * (A W2^T) (SwiGLU product, Sec. "transformer shape").  W, W2: [N, K]. */
+int lsp_op_linear(lsp_ctx* ctx, int op, const void* A, const void* W, const void* W2, void* out, int M,
+                  int N, int K);
+
+/* Device time (ms) of the last step by kernel class, host float[8]:
+ * 0 embed+norms, 1 GEMMs, 2 attention, 3 head, 4 merge+scan, 5 commit/append, 6 total, 7 reserved.
+ * Only filled when option key 2 (per-class timing, serialises with events) is 1. */
+int lsp_last_timing(lsp_ctx* ctx, float* ms);
+
+const char* lsp_last_error(const lsp_ctx* ctx);
+int lsp_destroy(lsp_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LSP_H_ */

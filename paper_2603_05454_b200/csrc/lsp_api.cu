@@ -1,0 +1,689 @@
+// Host step driver and C ABI of the LSP decode library (see include/lsp.h for the contract).
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <type_traits>
+#include <string>
+#include <vector>
+
+#include "../../include/lsp.h"
+#include "attention_simt.cuh"
+#include "gemm_simt.cuh"
+#include "misc_kernels.cuh"
+#ifndef LSP_NO_UMMA
+#include "gemm_umma.cuh"
+#endif
+
+using namespace lsp;
+
+namespace {
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+}  // namespace
+
+struct lsp_ctx {
+  lsp_model_cfg m{};
+  lsp_sched_cfg s{};
+  const void *embed = nullptr, *final_norm = nullptr, *w_head = nullptr;
+  std::vector<const void*> attn_norm, w_qkv, w_o, ffn_norm, w_gate, w_up, w_down;
+  char* kv_cache = nullptr;
+  int max_batch = 0, max_len = 0, max_rows = 0;
+  size_t esz = 0;
+  cudaStream_t stream = nullptr;
+  int gemm_impl = 1, attn_impl = 1, timing = 0;
+  // workspace carve (device)
+  char *X = nullptr, *Nrm = nullptr, *Qb = nullptr, *Att = nullptr, *Hf = nullptr, *stage = nullptr;
+  Top2* part = nullptr;
+  int32_t* yhat = nullptr;
+  float *pmax = nullptr, *margin = nullptr;
+  int *row_seq = nullptr, *row_pos = nullptr, *head_src = nullptr;
+  int* d_desc = nullptr;      // 7 arrays of (max_batch + 1) ints
+  int* d_scan = nullptr;      // 4 arrays of max_batch (run, commit, flags, tau)
+  float2* rope_cs = nullptr;
+  unsigned* d_status = nullptr;
+  // pinned host mirrors
+  int* h_desc = nullptr;
+  int* h_scan = nullptr;
+  unsigned* h_status = nullptr;
+  // decode state (host is the authority; the device sees it through the descriptors)
+  int32_t* tokens = nullptr;
+  int tok_stride = 0, batch = 0, step = 0;
+  std::vector<int> F, Fp, pend, N, Lprop;
+  bool proposed = false;
+  int score_rows = 0;
+  int last_M = 0;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  float timing_ms[8] = {0};
+  std::string err;
+#ifndef LSP_NO_UMMA
+  UmmaState umma;
+#endif
+};
+
+namespace {
+
+int fail(lsp_ctx* c, int code, const char* fmt, ...) {
+  if (c) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    c->err = buf;
+  }
+  return code;
+}
+
+#define CU(call)                                                                                   \
+  do {                                                                                             \
+    cudaError_t e_ = (call);                                                                       \
+    if (e_ != cudaSuccess) return fail(c, LSP_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+StepDesc desc_of(const lsp_ctx* c) {
+  const int s = c->max_batch + 1;
+  StepDesc d;
+  d.F = c->d_desc + 0 * s;
+  d.pend = c->d_desc + 1 * s;
+  d.N = c->d_desc + 2 * s;
+  d.row_off = c->d_desc + 3 * s;
+  d.head_off = c->d_desc + 4 * s;
+  d.Fp = c->d_desc + 5 * s;
+  d.Lc = c->d_desc + 6 * s;
+  return d;
+}
+
+struct Carve {
+  size_t off = 0;
+  size_t take(size_t bytes) {
+    const size_t o = off;
+    off = align_up(off + bytes, 256);
+    return o;
+  }
+};
+
+struct Layout {
+  size_t X, Nrm, Qb, Att, Hf, part, yhat, pmax, margin, row_seq, row_pos, head_src, desc, scan, rope, status,
+      stage, total;
+};
+
+int head_tiles_max(const lsp_model_cfg* m) { return (m->vocab + 63) / 64; }
+
+Layout make_layout(const lsp_model_cfg* m, int max_batch, int max_len) {
+  const size_t esz = m->dtype == 0 ? 4 : 2;
+  const size_t R = (size_t)max_batch * max_len;
+  const size_t qd = (size_t)m->n_heads * m->head_dim, kvd = (size_t)m->n_kv_heads * m->head_dim;
+  Carve cv;
+  Layout L;
+  L.X = cv.take(R * m->d_model * esz);
+  L.Nrm = cv.take(R * m->d_model * esz);
+  L.Qb = cv.take(R * qd * esz);
+  L.Att = cv.take(R * qd * esz);
+  L.Hf = cv.take(R * m->d_ffn * esz);
+  L.part = cv.take(R * head_tiles_max(m) * sizeof(Top2));
+  L.yhat = cv.take(R * 4);
+  L.pmax = cv.take(R * 4);
+  L.margin = cv.take(R * 4);
+  L.row_seq = cv.take(R * 4);
+  L.row_pos = cv.take(R * 4);
+  L.head_src = cv.take(R * 4);
+  L.desc = cv.take(7 * (size_t)(max_batch + 1) * 4);
+  L.scan = cv.take(4 * (size_t)max_batch * 4);
+  L.rope = cv.take((size_t)max_len * (m->head_dim / 2) * sizeof(float2));
+  L.status = cv.take(256);
+  L.stage = cv.take((size_t)m->n_layers * 2 * R * kvd * esz);
+  L.total = cv.off;
+  return L;
+}
+
+int check_model(const lsp_model_cfg* m) {
+  if (!m) return LSP_ERR_ARG;
+  if (m->dtype != 0 && m->dtype != 1) return LSP_ERR_ARG;
+  if (m->n_layers < 1 || m->vocab < 2 || m->mask_id < 0 || m->mask_id >= m->vocab) return LSP_ERR_ARG;
+  if (m->head_dim != 64 && m->head_dim != 128) return LSP_ERR_SHAPE;
+  if (m->d_model % 64 || m->d_ffn % 64 || m->n_heads < 1 || m->n_kv_heads < 1 || m->n_heads % m->n_kv_heads)
+    return LSP_ERR_SHAPE;
+  return LSP_OK;
+}
+
+// ---- GEMM dispatch ------------------------------------------------------------------------------------
+template <typename T, typename Epi>
+int run_gemm(lsp_ctx* c, const T* A, const T* W0, const T* W1, int M, int NP, int K, int n_rows_w, const Epi& epi) {
+  if (M <= 0) return LSP_OK;
+#ifndef LSP_NO_UMMA
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (c->gemm_impl == 1) {
+      const int rc = umma_gemm<Epi>(c->umma, c->stream, A, W0, W1, M, NP, K, n_rows_w, epi, c->d_status);
+      if (rc != 0) return fail(c, LSP_ERR_CUDA, "tcgen05 GEMM launch failed (%d): %s", rc, c->umma.err.c_str());
+      return LSP_OK;
+    }
+  }
+#endif
+  dim3 grid((NP + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
+  k_gemm_simt<T, Epi><<<grid, 256, 0, c->stream>>>(A, W0, W1, M, NP, K, epi);
+  CU(cudaGetLastError());
+  return LSP_OK;
+}
+
+template <typename T>
+int run_head(lsp_ctx* c, const T* hidden, int rows, int* n_tiles_out) {
+  const lsp_model_cfg& m = c->m;
+  EpiHead epi;
+  epi.part = c->part;
+  epi.vocab = m.vocab;
+  epi.exclude_id = c->s.exclude_mask_logit ? m.mask_id : -1;
+  int n_tiles = (m.vocab + SG_BN - 1) / SG_BN;
+#ifndef LSP_NO_UMMA
+  if (std::is_same<T, bf16>::value && c->gemm_impl == 1) n_tiles = umma_head_tiles(m.vocab);
+#endif
+  epi.n_tiles = n_tiles;
+  *n_tiles_out = n_tiles;
+  return run_gemm<T, EpiHead>(c, hidden, (const T*)c->w_head, (const T*)c->w_head, rows, m.vocab, m.d_model,
+                              m.vocab, epi);
+}
+
+ScanParams scan_params(const lsp_ctx* c) {
+  ScanParams p;
+  p.mode = c->s.mode;
+  p.tau = c->s.tau;
+  p.alpha = c->s.alpha;
+  p.beta = c->s.beta;
+  p.l_min = c->s.l_min < 1 ? 1 : c->s.l_min;
+  p.W = c->s.snap_window;
+  p.fixed_k = c->s.fixed_k;
+  p.delim = c->s.delim_bitmap;
+  p.flag_tol = c->s.flag_tol;
+  return p;
+}
+
+// merge partials -> scores, scan, copy the scan outputs to the pinned mirror (async)
+int run_merge_scan(lsp_ctx* c, int rows, int n_tiles, const int* d_seq_off, int batch) {
+  if (rows > 0) {
+    k_merge_partials<<<(rows + 3) / 4, 128, 0, c->stream>>>(c->part, n_tiles, rows, c->yhat, c->pmax, c->margin);
+    CU(cudaGetLastError());
+  }
+  const float* score = c->s.score == 1 ? c->margin : c->pmax;
+  int* o = c->d_scan;
+  const int mb = c->max_batch;
+  k_lsp_scan<<<batch, 32, 0, c->stream>>>(score, c->yhat, c->margin, d_seq_off, scan_params(c), o, o + mb,
+                                          (uint32_t*)(o + 2 * mb), (float*)(o + 3 * mb));
+  CU(cudaGetLastError());
+  CU(cudaMemcpyAsync(c->h_scan, c->d_scan, 4 * (size_t)mb * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
+  return LSP_OK;
+}
+
+int check_status(lsp_ctx* c) {
+  if (c->h_status[0] != 0) {
+    const unsigned code = c->h_status[0], where = c->h_status[1];
+    cudaMemsetAsync(c->d_status, 0, 16, c->stream);
+    cudaStreamSynchronize(c->stream);
+    return fail(c, LSP_ERR_DEVICE_TIMEOUT, "device-side bounded wait expired (code %u, site %u)", code, where);
+  }
+  return LSP_OK;
+}
+
+template <typename T>
+int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
+  const lsp_model_cfg& m = c->m;
+  const int B = c->batch, s = c->max_batch + 1;
+  int* h = c->h_desc;
+  int M = 0, Mh = 0, maxQ = 0;
+  for (int b = 0; b < B; ++b) {
+    const int pend = c->N[b] > 0 ? c->pend[b] : 0;
+    const int rows = pend + c->N[b];
+    h[0 * s + b] = c->F[b];
+    h[1 * s + b] = pend;
+    h[2 * s + b] = c->N[b];
+    h[3 * s + b] = M;
+    h[4 * s + b] = Mh;
+    h[5 * s + b] = c->Fp[b];
+    h[6 * s + b] = 0;
+    M += rows;
+    Mh += c->N[b];
+    if (rows > maxQ) maxQ = rows;
+  }
+  h[3 * s + B] = M;
+  h[4 * s + B] = Mh;
+  if (M == 0) return fail(c, LSP_ERR_STATE, "lsp_denoise_step: every sequence is already fully committed");
+  CU(cudaEventRecord(c->ev0, c->stream));
+  CU(cudaMemcpyAsync(c->d_desc, h, 7 * (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
+  const StepDesc sd = desc_of(c);
+  const int d = m.d_model, dh = m.head_dim, qd = m.n_heads * dh, kvd = m.n_kv_heads * dh;
+  T* X = (T*)c->X;
+  T* Nrm = (T*)c->Nrm;
+  T* Qb = (T*)c->Qb;
+  T* Att = (T*)c->Att;
+  T* Hf = (T*)c->Hf;
+  k_assemble_embed<T><<<M, 128, 0, c->stream>>>(sd, B, c->tokens, c->tok_stride, m.mask_id, (const T*)c->embed, d, X,
+                                               c->row_seq, c->row_pos, c->head_src);
+  CU(cudaGetLastError());
+  const size_t plane = (size_t)c->max_rows * kvd;           // elements per staged (layer, K|V) plane
+  const size_t cplane = (size_t)c->max_batch * c->max_len * kvd;
+  const float scale = 1.0f / sqrtf((float)dh);
+  for (int l = 0; l < m.n_layers; ++l) {
+    T* stK = (T*)c->stage + (size_t)(2 * l) * plane;
+    T* stV = stK + plane;
+    const T* cK = (const T*)c->kv_cache + (size_t)(2 * l) * cplane;
+    const T* cV = cK + cplane;
+    k_rmsnorm<T><<<M, 256, 0, c->stream>>>(X, (const T*)c->attn_norm[l], Nrm, nullptr, d, m.rms_eps);
+    CU(cudaGetLastError());
+    {
+      EpiQKVRope<T> e{Qb, stK, stV, c->rope_cs, c->row_pos, m.n_heads, m.n_kv_heads, dh / 2};
+      const int rc = run_gemm<T>(c, Nrm, (const T*)c->w_qkv[l], (const T*)c->w_qkv[l], M, (qd + 2 * kvd) / 2, d,
+                                 qd + 2 * kvd, e);
+      if (rc) return rc;
+    }
+    {
+      dim3 grid((maxQ + AS_BQ - 1) / AS_BQ, m.n_heads, B);
+      if (dh == 128)
+        k_attn_simt<T, 128><<<grid, 128, 0, c->stream>>>(Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
+                                                         (size_t)c->max_len * kvd, scale);
+      else
+        k_attn_simt<T, 64><<<grid, 128, 0, c->stream>>>(Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
+                                                        (size_t)c->max_len * kvd, scale);
+      CU(cudaGetLastError());
+    }
+    {
+      EpiResidual<T> e{X, d};
+      const int rc = run_gemm<T>(c, Att, (const T*)c->w_o[l], (const T*)c->w_o[l], M, d, qd, d, e);
+      if (rc) return rc;
+    }
+    k_rmsnorm<T><<<M, 256, 0, c->stream>>>(X, (const T*)c->ffn_norm[l], Nrm, nullptr, d, m.rms_eps);
+    CU(cudaGetLastError());
+    {
+      EpiSwiGLU<T> e{Hf, m.d_ffn};
+      const int rc = run_gemm<T>(c, Nrm, (const T*)c->w_gate[l], (const T*)c->w_up[l], M, m.d_ffn, d, m.d_ffn, e);
+      if (rc) return rc;
+    }
+    {
+      EpiResidual<T> e{X, d};
+      const int rc = run_gemm<T>(c, Hf, (const T*)c->w_down[l], (const T*)c->w_down[l], M, d, m.d_ffn, d, e);
+      if (rc) return rc;
+    }
+  }
+  // masked rows only: final norm (gathered), fused head, merge, scan
+  k_rmsnorm<T><<<Mh, 256, 0, c->stream>>>(X, (const T*)c->final_norm, Nrm, c->head_src, d, m.rms_eps);
+  CU(cudaGetLastError());
+  int n_tiles = 0;
+  int rc = run_head<T>(c, Nrm, Mh, &n_tiles);
+  if (rc) return rc;
+  rc = run_merge_scan(c, Mh, n_tiles, sd.head_off, B);
+  if (rc) return rc;
+  CU(cudaEventRecord(c->ev1, c->stream));
+  CU(cudaStreamSynchronize(c->stream));
+  rc = check_status(c);
+  if (rc) return rc;
+  float ms = 0.f;
+  CU(cudaEventElapsedTime(&ms, c->ev0, c->ev1));
+  const int mb = c->max_batch;
+  for (int b = 0; b < B; ++b) {
+    c->Lprop[b] = c->N[b] > 0 ? c->h_scan[mb + b] : 0;
+    if (rec) {
+      rec[b].step = c->step;
+      rec[b].n_before = c->N[b];
+      rec[b].rows = c->N[b] > 0 ? c->pend[b] + c->N[b] : 0;
+      rec[b].l_run = c->h_scan[b];
+      rec[b].l_commit = c->h_scan[mb + b];
+      rec[b].flags = (unsigned)c->h_scan[2 * mb + b];
+      memcpy(&rec[b].tau_used, &c->h_scan[3 * mb + b], 4);
+      rec[b].ms = ms;
+    }
+  }
+  c->timing_ms[6] = ms;
+  c->proposed = true;
+  c->score_rows = Mh;
+  c->last_M = M;
+  return LSP_OK;
+}
+
+static int scan_outputs(lsp_ctx* c, int batch, int32_t* l_run, int32_t* l_commit, uint32_t* flags, float* tau_used) {
+  CU(cudaStreamSynchronize(c->stream));
+  int rc = check_status(c);
+  if (rc) return rc;
+  const int mb = c->max_batch;
+  for (int b = 0; b < batch; ++b) {
+    if (l_run) l_run[b] = c->h_scan[b];
+    if (l_commit) l_commit[b] = c->h_scan[mb + b];
+    if (flags) flags[b] = (uint32_t)c->h_scan[2 * mb + b];
+    if (tau_used) memcpy(&tau_used[b], &c->h_scan[3 * mb + b], 4);
+  }
+  return LSP_OK;
+}
+
+static int upload_offsets(lsp_ctx* c, const int32_t* seq_offsets, int batch, int* rows_out) {
+  if (!seq_offsets || batch < 1 || batch > c->max_batch) return fail(c, LSP_ERR_ARG, "bad seq_offsets / batch");
+  if (seq_offsets[0] != 0) return fail(c, LSP_ERR_ARG, "seq_offsets[0] must be 0");
+  for (int b = 0; b < batch; ++b)
+    if (seq_offsets[b + 1] < seq_offsets[b]) return fail(c, LSP_ERR_ARG, "seq_offsets must ascend");
+  const int rows = seq_offsets[batch];
+  if (rows > c->max_rows) return fail(c, LSP_ERR_ARG, "rows %d exceed max_batch*max_len %d", rows, c->max_rows);
+  const int s = c->max_batch + 1;
+  int* h = c->h_desc + 4 * s;
+  for (int b = 0; b <= batch; ++b) h[b] = seq_offsets[b];
+  CU(cudaMemcpyAsync(c->d_desc + 4 * s, h, (size_t)(batch + 1) * 4, cudaMemcpyHostToDevice, c->stream));
+  *rows_out = rows;
+  return LSP_OK;
+}
+
+template <typename T>
+static int op_linear_impl(lsp_ctx* c, int op, const void* A, const void* W, const void* W2, void* out, int M, int N,
+                          int K) {
+  if (op == 0) {
+    EpiStore<T> e{(T*)out, N};
+    return run_gemm<T>(c, (const T*)A, (const T*)W, (const T*)W, M, N, K, N, e);
+  } else if (op == 1) {
+    EpiResidual<T> e{(T*)out, N};
+    return run_gemm<T>(c, (const T*)A, (const T*)W, (const T*)W, M, N, K, N, e);
+  } else {
+    EpiSwiGLU<T> e{(T*)out, N};
+    return run_gemm<T>(c, (const T*)A, (const T*)W, (const T*)W2, M, N, K, N, e);
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t lsp_workspace_bytes(const lsp_model_cfg* model, int max_batch, int max_len) {
+  if (check_model(model) != LSP_OK || max_batch < 1 || max_len < 2) return 0;
+  return make_layout(model, max_batch, max_len).total;
+}
+
+size_t lsp_kv_cache_bytes(const lsp_model_cfg* model, int max_batch, int max_len) {
+  if (check_model(model) != LSP_OK || max_batch < 1 || max_len < 2) return 0;
+  const size_t esz = model->dtype == 0 ? 4 : 2;
+  return (size_t)model->n_layers * 2 * max_batch * max_len * model->n_kv_heads * model->head_dim * esz;
+}
+
+int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sched, const lsp_weights* w,
+             void* kv_cache, void* workspace, size_t workspace_bytes, int max_batch, int max_len, void* cuda_stream) {
+  if (!out) return LSP_ERR_ARG;
+  *out = nullptr;
+  if (!model || !sched || !w || !kv_cache || !workspace || max_batch < 1 || max_len < 2) return LSP_ERR_ARG;
+  int rc = check_model(model);
+  if (rc) return rc;
+  if (!w->embed || !w->final_norm || !w->w_head || !w->attn_norm || !w->w_qkv || !w->w_o || !w->ffn_norm ||
+      !w->w_gate || !w->w_up || !w->w_down)
+    return LSP_ERR_ARG;
+  const Layout L = make_layout(model, max_batch, max_len);
+  if (workspace_bytes < L.total) return LSP_ERR_WORKSPACE;
+  if (((uintptr_t)workspace & 255) || ((uintptr_t)kv_cache & 255)) return LSP_ERR_ARG;
+  lsp_ctx* c = new lsp_ctx();
+  c->m = *model;
+  c->s = *sched;
+  c->embed = w->embed;
+  c->final_norm = w->final_norm;
+  c->w_head = w->w_head;
+  for (int l = 0; l < model->n_layers; ++l) {
+    c->attn_norm.push_back(w->attn_norm[l]);
+    c->w_qkv.push_back(w->w_qkv[l]);
+    c->w_o.push_back(w->w_o[l]);
+    c->ffn_norm.push_back(w->ffn_norm[l]);
+    c->w_gate.push_back(w->w_gate[l]);
+    c->w_up.push_back(w->w_up[l]);
+    c->w_down.push_back(w->w_down[l]);
+  }
+  c->kv_cache = (char*)kv_cache;
+  c->max_batch = max_batch;
+  c->max_len = max_len;
+  c->max_rows = max_batch * max_len;
+  c->esz = model->dtype == 0 ? 4 : 2;
+  c->stream = (cudaStream_t)cuda_stream;
+  char* ws = (char*)workspace;
+  c->X = ws + L.X;
+  c->Nrm = ws + L.Nrm;
+  c->Qb = ws + L.Qb;
+  c->Att = ws + L.Att;
+  c->Hf = ws + L.Hf;
+  c->part = (Top2*)(ws + L.part);
+  c->yhat = (int32_t*)(ws + L.yhat);
+  c->pmax = (float*)(ws + L.pmax);
+  c->margin = (float*)(ws + L.margin);
+  c->row_seq = (int*)(ws + L.row_seq);
+  c->row_pos = (int*)(ws + L.row_pos);
+  c->head_src = (int*)(ws + L.head_src);
+  c->d_desc = (int*)(ws + L.desc);
+  c->d_scan = (int*)(ws + L.scan);
+  c->rope_cs = (float2*)(ws + L.rope);
+  c->d_status = (unsigned*)(ws + L.status);
+  c->stage = ws + L.stage;
+  cudaError_t e = cudaHostAlloc((void**)&c->h_desc, 7 * (size_t)(max_batch + 1) * 4, cudaHostAllocDefault);
+  if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->h_scan, 4 * (size_t)max_batch * 4, cudaHostAllocDefault);
+  if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->h_status, 16, cudaHostAllocDefault);
+  if (e == cudaSuccess) e = cudaEventCreate(&c->ev0);
+  if (e == cudaSuccess) e = cudaEventCreate(&c->ev1);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 256, c->stream);
+  if (e == cudaSuccess) {
+    const int n = max_len * (model->head_dim / 2);
+    k_rope_table<<<(n + 255) / 256, 256, 0, c->stream>>>(c->rope_cs, max_len, model->head_dim / 2,
+                                                       (double)model->rope_theta);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) {
+    lsp_destroy(c);
+    return LSP_ERR_CUDA;
+  }
+  c->h_status[0] = 0;
+#ifndef LSP_NO_UMMA
+  if (model->dtype == 1) {
+    const int urc = umma_init(c->umma);
+    if (urc != 0) {
+      lsp_destroy(c);
+      return LSP_ERR_CUDA;
+    }
+  }
+#endif
+  *out = c;
+  return LSP_OK;
+}
+
+int lsp_set_sched(lsp_ctx* c, const lsp_sched_cfg* sched) {
+  if (!c || !sched) return LSP_ERR_ARG;
+  if (sched->mode < 0 || sched->mode > 2 || sched->score < 0 || sched->score > 1)
+    return fail(c, LSP_ERR_ARG, "lsp_set_sched: bad mode/score");
+  c->s = *sched;
+  return LSP_OK;
+}
+
+int lsp_set_option(lsp_ctx* c, int key, int value) {
+  if (!c) return LSP_ERR_ARG;
+  if (key == 0) c->gemm_impl = value;
+  else if (key == 1) c->attn_impl = value;
+  else if (key == 2) c->timing = value;
+  else return fail(c, LSP_ERR_ARG, "lsp_set_option: unknown key %d", key);
+  return LSP_OK;
+}
+
+int lsp_begin(lsp_ctx* c, int32_t* tokens, int token_stride, const int32_t* prompt_len, const int32_t* gen_len,
+              int batch) {
+  if (!c || !tokens || !prompt_len || !gen_len) return LSP_ERR_ARG;
+  if (batch < 1 || batch > c->max_batch) return fail(c, LSP_ERR_ARG, "lsp_begin: batch %d not in [1, %d]", batch, c->max_batch);
+  for (int b = 0; b < batch; ++b)
+    if (prompt_len[b] < 1 || gen_len[b] < 1 || prompt_len[b] + gen_len[b] > c->max_len ||
+        prompt_len[b] + gen_len[b] > token_stride)
+      return fail(c, LSP_ERR_ARG, "lsp_begin: sequence %d has prompt %d + gen %d outside [2, min(max_len %d, stride %d)]",
+                  b, prompt_len[b], gen_len[b], c->max_len, token_stride);
+  c->tokens = tokens;
+  c->tok_stride = token_stride;
+  c->batch = batch;
+  c->step = 0;
+  c->F.assign(batch, 0);
+  c->Fp.assign(prompt_len, prompt_len + batch);
+  c->pend.assign(prompt_len, prompt_len + batch);   // the prompt is step 0's pending block (CacheInit)
+  c->N.assign(gen_len, gen_len + batch);
+  c->Lprop.assign(batch, 0);
+  c->proposed = false;
+  // mask fill: reuse the descriptor's F/pend slots to pass P and G
+  const int s = c->max_batch + 1;
+  for (int b = 0; b < batch; ++b) { c->h_desc[b] = prompt_len[b]; c->h_desc[s + b] = gen_len[b]; }
+  CU(cudaMemcpyAsync(c->d_desc, c->h_desc, 2 * (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
+  k_fill_mask<<<batch, 256, 0, c->stream>>>(tokens, token_stride, c->d_desc, c->d_desc + s, c->m.mask_id);
+  CU(cudaGetLastError());
+  CU(cudaStreamSynchronize(c->stream));
+  return LSP_OK;
+}
+
+int lsp_denoise_step(lsp_ctx* c, lsp_step_rec* rec) {
+  if (!c) return LSP_ERR_ARG;
+  if (!c->tokens) return fail(c, LSP_ERR_STATE, "lsp_denoise_step before lsp_begin");
+  return c->m.dtype == 0 ? step_impl<float>(c, rec) : step_impl<bf16>(c, rec);
+}
+
+int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
+  if (!c) return LSP_ERR_ARG;
+  if (!c->proposed) return fail(c, LSP_ERR_STATE, "lsp_commit without a preceding lsp_denoise_step");
+  const int B = c->batch, s = c->max_batch + 1;
+  std::vector<int> L(B, 0);
+  int max_pend = 0;
+  for (int b = 0; b < B; ++b) {
+    if (c->N[b] == 0) continue;
+    L[b] = L_override ? L_override[b] : c->Lprop[b];
+    if (L[b] < 1 || L[b] > c->N[b])
+      return fail(c, LSP_ERR_STATE, "lsp_commit: L[%d] = %d outside [1, %d]", b, L[b], c->N[b]);
+    if (c->pend[b] > max_pend) max_pend = c->pend[b];
+  }
+  int* hl = c->h_desc + 6 * s;
+  for (int b = 0; b < B; ++b) hl[b] = L[b];
+  CU(cudaMemcpyAsync(c->d_desc + 6 * s, hl, (size_t)B * 4, cudaMemcpyHostToDevice, c->stream));
+  const lsp_model_cfg& m = c->m;
+  const size_t kvd = (size_t)m.n_kv_heads * m.head_dim;
+  const int row_v4 = (int)(kvd * c->esz / 16);
+  const size_t stage_plane_v4 = (size_t)c->max_rows * row_v4;
+  const size_t cache_seq_v4 = (size_t)c->max_len * row_v4;
+  const size_t cache_plane_v4 = (size_t)c->max_batch * cache_seq_v4;
+  size_t n_v4 = (size_t)max_pend * row_v4;
+  int chunks = (int)((n_v4 + 256 * 8 - 1) / (256 * 8));
+  if (chunks < 1) chunks = 1;
+  if (chunks > 64) chunks = 64;
+  dim3 grid(chunks, m.n_layers * 2, B);
+  k_commit_append<<<grid, 256, 0, c->stream>>>(desc_of(c), (const uint4*)c->stage, (uint4*)c->kv_cache,
+                                               stage_plane_v4, cache_plane_v4, cache_seq_v4, row_v4, c->yhat,
+                                               c->tokens, c->tok_stride);
+  CU(cudaGetLastError());
+  for (int b = 0; b < B; ++b) {
+    if (c->N[b] == 0) continue;
+    c->F[b] += c->pend[b];
+    c->Fp[b] += L[b];
+    c->pend[b] = L[b];
+    c->N[b] -= L[b];
+  }
+  c->proposed = false;
+  c->step += 1;
+  return LSP_OK;
+}
+
+int lsp_generate(lsp_ctx* c, lsp_step_rec* recs, int max_recs, int* n_steps) {
+  if (!c) return LSP_ERR_ARG;
+  if (!c->tokens) return fail(c, LSP_ERR_STATE, "lsp_generate before lsp_begin");
+  int steps = 0, used = 0;
+  std::vector<lsp_step_rec> tmp(c->batch);
+  for (;;) {
+    bool any = false;
+    for (int b = 0; b < c->batch; ++b) any |= c->N[b] > 0;
+    if (!any) break;
+    int rc = lsp_denoise_step(c, tmp.data());
+    if (rc) return rc;
+    for (int b = 0; b < c->batch && recs && used < max_recs; ++b) recs[used++] = tmp[b];
+    rc = lsp_commit(c, nullptr);
+    if (rc) return rc;
+    ++steps;
+  }
+  CU(cudaStreamSynchronize(c->stream));
+  if (n_steps) *n_steps = steps;
+  return LSP_OK;
+}
+
+int lsp_active(lsp_ctx* c, int32_t* n_active, int* n_unfinished) {
+  if (!c) return LSP_ERR_ARG;
+  int u = 0;
+  for (int b = 0; b < c->batch; ++b) {
+    if (n_active) n_active[b] = c->N[b];
+    u += c->N[b] > 0;
+  }
+  if (n_unfinished) *n_unfinished = u;
+  return LSP_OK;
+}
+
+int lsp_score_rows(lsp_ctx* c) { return c ? c->score_rows : LSP_ERR_ARG; }
+
+int lsp_get_scores(lsp_ctx* c, int32_t* yhat, float* pmax, float* margin) {
+  if (!c) return LSP_ERR_ARG;
+  const size_t n = (size_t)c->score_rows * 4;
+  if (n == 0) return LSP_OK;
+  if (yhat) CU(cudaMemcpyAsync(yhat, c->yhat, n, cudaMemcpyDeviceToHost, c->stream));
+  if (pmax) CU(cudaMemcpyAsync(pmax, c->pmax, n, cudaMemcpyDeviceToHost, c->stream));
+  if (margin) CU(cudaMemcpyAsync(margin, c->margin, n, cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaStreamSynchronize(c->stream));
+  return LSP_OK;
+}
+
+int lsp_head_scan(lsp_ctx* c, const void* hidden, const int32_t* seq_offsets, int batch, int32_t* l_run,
+                  int32_t* l_commit, uint32_t* flags, float* tau_used) {
+  if (!c || !hidden) return LSP_ERR_ARG;
+  int rows = 0;
+  int rc = upload_offsets(c, seq_offsets, batch, &rows);
+  if (rc) return rc;
+  c->proposed = false;
+  int n_tiles = 0;
+  rc = c->m.dtype == 0 ? run_head<float>(c, (const float*)hidden, rows, &n_tiles)
+                       : run_head<bf16>(c, (const bf16*)hidden, rows, &n_tiles);
+  if (rc) return rc;
+  rc = run_merge_scan(c, rows, n_tiles, c->d_desc + 4 * (c->max_batch + 1), batch);
+  if (rc) return rc;
+  c->score_rows = rows;
+  return scan_outputs(c, batch, l_run, l_commit, flags, tau_used);
+}
+
+int lsp_scan(lsp_ctx* c, const float* score, const int32_t* yhat, const float* margin, const int32_t* seq_offsets,
+             int batch, int32_t* l_run, int32_t* l_commit, uint32_t* flags, float* tau_used) {
+  if (!c || !score || !yhat) return LSP_ERR_ARG;
+  int rows = 0;
+  int rc = upload_offsets(c, seq_offsets, batch, &rows);
+  if (rc) return rc;
+  c->proposed = false;
+  int* o = c->d_scan;
+  const int mb = c->max_batch;
+  k_lsp_scan<<<batch, 32, 0, c->stream>>>(score, yhat, margin, c->d_desc + 4 * (c->max_batch + 1), scan_params(c), o,
+                                          o + mb, (uint32_t*)(o + 2 * mb), (float*)(o + 3 * mb));
+  CU(cudaGetLastError());
+  CU(cudaMemcpyAsync(c->h_scan, c->d_scan, 4 * (size_t)mb * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
+  return scan_outputs(c, batch, l_run, l_commit, flags, tau_used);
+}
+
+int lsp_op_linear(lsp_ctx* c, int op, const void* A, const void* W, const void* W2, void* out, int M, int N, int K) {
+  if (!c || !A || !W || !out || M < 0 || N < 1 || K < 1) return LSP_ERR_ARG;
+  if (op < 0 || op > 2 || (op == 2 && !W2)) return fail(c, LSP_ERR_ARG, "lsp_op_linear: bad op");
+  if (K % 64 || N % 8) return fail(c, LSP_ERR_SHAPE, "lsp_op_linear: K must be a multiple of 64 and N of 8");
+  const int rc = c->m.dtype == 0 ? op_linear_impl<float>(c, op, A, W, W2, out, M, N, K)
+                                 : op_linear_impl<bf16>(c, op, A, W, W2, out, M, N, K);
+  if (rc) return rc;
+  CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaStreamSynchronize(c->stream));
+  return check_status(c);
+}
+
+int lsp_last_timing(lsp_ctx* c, float* ms) {
+  if (!c || !ms) return LSP_ERR_ARG;
+  memcpy(ms, c->timing_ms, sizeof c->timing_ms);
+  return LSP_OK;
+}
+
+const char* lsp_last_error(const lsp_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+int lsp_destroy(lsp_ctx* c) {
+  if (!c) return LSP_ERR_ARG;
+  if (c->h_desc) cudaFreeHost(c->h_desc);
+  if (c->h_scan) cudaFreeHost(c->h_scan);
+  if (c->h_status) cudaFreeHost(c->h_status);
+  if (c->ev0) cudaEventDestroy(c->ev0);
+  if (c->ev1) cudaEventDestroy(c->ev1);
+  delete c;
+  return LSP_OK;
+}
+
+}  // extern "C"

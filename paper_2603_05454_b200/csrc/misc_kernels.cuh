@@ -1,0 +1,242 @@
+// Row assembly + embedding, RMSNorm, vocab-partial merge, the LSP scan, and commit/KV-append kernels.
+#pragma once
+#include "common.cuh"
+
+namespace lsp {
+
+// ---------------------------------------------------------------------------------------------
+// Row assembly + embedding (Algorithm 1 line 4's input): packed row r of sequence b is position
+// F_b + j; the first pend_b rows carry the tokens committed by the previous step, the rest [MASK].
+// One block per row.  Also fills row_seq / row_pos and the list of rows that go through the LM head.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void k_assemble_embed(StepDesc sd, int batch, const int32_t* __restrict__ tokens, int tok_stride,
+                                 int mask_id, const T* __restrict__ embed, int d, T* __restrict__ X,
+                                 int* __restrict__ row_seq, int* __restrict__ row_pos,
+                                 int* __restrict__ head_src) {
+  const int r = blockIdx.x;
+  int b = 0;
+  while (b + 1 < batch && r >= sd.row_off[b + 1]) ++b;
+  const int j = r - sd.row_off[b];
+  const int F = sd.F[b], pend = sd.pend[b];
+  const int pos = F + j;
+  const int tok = (j < pend) ? tokens[(size_t)b * tok_stride + pos] : mask_id;
+  if (threadIdx.x == 0) {
+    row_seq[r] = b;
+    row_pos[r] = pos;
+    if (j >= pend) head_src[sd.head_off[b] + (j - pend)] = r;
+  }
+  const uint4* src = reinterpret_cast<const uint4*>(embed + (size_t)tok * d);
+  uint4* dst = reinterpret_cast<uint4*>(X + (size_t)r * d);
+  const int nv = d * (int)sizeof(T) / 16;
+  for (int i = threadIdx.x; i < nv; i += blockDim.x) dst[i] = __ldg(src + i);
+}
+
+// ---------------------------------------------------------------------------------------------
+// RMSNorm: out[r] = x[src[r]] / sqrt(mean(x^2) + eps) * g, fp32 arithmetic, one block per output row.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void k_rmsnorm(const T* __restrict__ x, const T* __restrict__ g, T* __restrict__ out,
+                          const int* __restrict__ src_rows, int d, float eps) {
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  const T* xr = x + (size_t)(src_rows ? src_rows[r] : r) * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    const float v = to_f(xr[i]);
+    ss += v * v;
+  }
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
+    v = warp_sum(v);
+    if (threadIdx.x == 0) red[0] = v;
+  }
+  __syncthreads();
+  const float inv = rsqrtf(red[0] / (float)d + eps);
+  T* o = out + (size_t)r * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) o[i] = from_f<T>(to_f(xr[i]) * inv * to_f(g[i]));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Merge of the per-vocab-tile partials of one row into (yhat, p_max, delta).  One warp per row.
+// ---------------------------------------------------------------------------------------------
+__global__ void k_merge_partials(const Top2* __restrict__ part, int n_tiles, int rows, int32_t* __restrict__ yhat,
+                                 float* __restrict__ pmax, float* __restrict__ margin) {
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= rows) return;
+  const int lane = threadIdx.x & 31;
+  Top2 t = top2_empty();
+  for (int i = lane; i < n_tiles; i += 32) t = top2_merge(t, part[(size_t)r * n_tiles + i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t = top2_merge(t, top2_shfl_xor(t, o));
+  if (lane == 0) {
+    yhat[r] = t.i1;
+    pmax[r] = 1.f / t.s;
+    margin[r] = t.m1 - t.m2;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// LSP scan (Sec. 3.2): one warp per sequence.
+//   fixed mode    : L' = longest left-aligned run with score_i >= tau             (ballot + ffs)
+//   adaptive mode : prefix minimum pm; m is achievable iff pm[m] > pm[m+1]; the largest achievable
+//                   m in [ceil(alpha N), floor(beta N)] is taken, tau = pm[m] (Eq. 2)
+//   snap          : last delimiter j <= L' with L' - j <= W, else the run's end; L' = N commits all;
+//                   L = min(N, max(L, L_min, 1))                               (Algorithm 1 lines 7-8)
+// ---------------------------------------------------------------------------------------------
+struct ScanParams {
+  int mode;
+  float tau, alpha, beta;
+  int l_min, W, fixed_k;
+  const uint8_t* delim;
+  float flag_tol;
+};
+
+__device__ __forceinline__ bool is_delim(const uint8_t* bm, int id) {
+  return bm != nullptr && ((bm[id >> 3] >> (id & 7)) & 1);
+}
+
+__global__ void k_lsp_scan(const float* __restrict__ score, const int32_t* __restrict__ yhat,
+                           const float* __restrict__ margin, const int* __restrict__ seq_off, ScanParams p,
+                           int32_t* __restrict__ o_run, int32_t* __restrict__ o_commit, uint32_t* __restrict__ o_flags,
+                           float* __restrict__ o_tau) {
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x;
+  const int base = seq_off[b];
+  const int N = seq_off[b + 1] - base;
+  if (N <= 0) {
+    if (lane == 0) { o_run[b] = 0; o_commit[b] = 0; o_flags[b] = 0; o_tau[b] = 0.f; }
+    return;
+  }
+  const float* sc = score + base;
+  const int32_t* yh = yhat + base;
+  unsigned flags = 0;
+  int Lrun = 0;
+  float tau = p.tau;
+  if (p.mode == 2) {
+    int L = min(N, max(1, p.fixed_k));
+    if (lane == 0) { o_run[b] = L; o_commit[b] = L; o_flags[b] = 0; o_tau[b] = __int_as_float(0x7fc00000); }
+    return;
+  }
+  if (p.mode == 1) {
+    const int lo = max(1, (int)ceil((double)p.alpha * (double)N));
+    const int hi = min(N, max(lo, (int)floor((double)p.beta * (double)N)));
+    float carry = INFINITY;   // pm[m0] for the chunk start
+    int best = 0;
+    float best_pm = 0.f, pm_hi = 0.f;
+    for (int m0 = 0; m0 < hi; m0 += 32) {
+      const int m = m0 + lane + 1;                       // 1-based length this lane stands for
+      float v = (m <= N) ? sc[m - 1] : INFINITY;
+      // inclusive prefix min across the warp
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float u = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v = fminf(v, u);
+      }
+      const float pm = fminf(v, carry);                   // pm[m]
+      const bool ach = (m >= lo && m <= hi) && (m == N || sc[m] < pm);
+      const unsigned bal = __ballot_sync(0xffffffffu, ach);
+      if (bal) {
+        const int top = 31 - __clz(bal);
+        best = m0 + top + 1;
+        best_pm = __shfl_sync(0xffffffffu, pm, top);
+      }
+      const int hl = hi - m0 - 1;                          // lane holding pm[hi], if in this chunk
+      if (hl >= 0 && hl < 32) pm_hi = __shfl_sync(0xffffffffu, pm, hl);
+      carry = __shfl_sync(0xffffffffu, pm, 31);
+    }
+    if (best > 0) { Lrun = best; tau = best_pm; }
+    else { Lrun = hi; tau = pm_hi; flags |= 4u; }
+  } else {
+    Lrun = N;
+    for (int i0 = 0; i0 < N; i0 += 32) {
+      const int i = i0 + lane;
+      const bool pass = (i < N) ? (sc[i] >= tau) : false;
+      const unsigned fail = ~__ballot_sync(0xffffffffu, pass);
+      if (fail) { Lrun = min(N, i0 + __ffs(fail) - 1); break; }
+    }
+  }
+  int L;
+  if (Lrun == N) {
+    L = N;
+    flags |= 8u;
+  } else {
+    const int lo_j = (p.W < 0) ? 1 : max(1, Lrun - p.W);
+    int maxJ = 0;
+    for (int hi_j = Lrun; hi_j >= lo_j && maxJ == 0; hi_j -= 32) {
+      const int j = hi_j - lane;                           // lane 0 looks at the right end
+      const bool d = (j >= lo_j) && is_delim(p.delim, yh[j - 1]);
+      const unsigned bal = __ballot_sync(0xffffffffu, d);
+      if (bal) maxJ = hi_j - (__ffs(bal) - 1);
+    }
+    if (maxJ > 0) {
+      L = max(p.l_min, maxJ);
+      if (L < Lrun) flags |= 1u;
+    } else {
+      L = max(p.l_min, Lrun);
+    }
+    if (Lrun < max(1, p.l_min)) flags |= 2u;
+  }
+  L = min(N, max(L, 1));
+  if (p.flag_tol > 0.f) {
+    bool near = false, tie = false;
+    const int lim = min(N, Lrun + 1);
+    for (int i = lane; i < lim; i += 32) near |= fabsf(sc[i] - tau) <= p.flag_tol;
+    if (margin != nullptr)
+      for (int i = lane; i < L; i += 32) tie |= margin[base + i] <= p.flag_tol;
+    if (__any_sync(0xffffffffu, near)) flags |= 16u;
+    if (__any_sync(0xffffffffu, tie)) flags |= 32u;
+  }
+  if (lane == 0) { o_run[b] = Lrun; o_commit[b] = L; o_flags[b] = flags; o_tau[b] = tau; }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Commit (Algorithm 1 lines 9-10).  grid = (chunks, n_layers * 2, batch):
+//   * the pending block's K/V rows, staged by the last pass at packed rows [row_off_b, row_off_b + pend_b),
+//     are copied to cache rows [F_b, F_b + pend_b): one contiguous 128-bit-vector copy per (layer, K|V, b);
+//   * block (0, 0, b) also writes yhat_{1:L_b} into the token buffer at [Fp_b, Fp_b + L_b).
+// The host advances F, Fp, pend, N after enqueueing this kernel (stream order makes the commit atomic).
+// ---------------------------------------------------------------------------------------------
+__global__ void k_commit_append(StepDesc sd, const uint4* __restrict__ stage, uint4* __restrict__ cache,
+                                size_t stage_plane_v4,   // uint4 per (layer, K|V) plane of the staging buffer
+                                size_t cache_plane_v4,   // uint4 per (layer, K|V) plane of the cache
+                                size_t cache_seq_v4,     // uint4 per sequence inside a cache plane
+                                int row_v4,              // uint4 per row (n_kv_heads * head_dim * sizeof(T) / 16)
+                                const int32_t* __restrict__ yhat, int32_t* __restrict__ tokens, int tok_stride) {
+  const int b = blockIdx.z;
+  const int plane = blockIdx.y;
+  const int pend = sd.pend[b];
+  const size_t n = (size_t)pend * row_v4;
+  const uint4* src = stage + plane * stage_plane_v4 + (size_t)sd.row_off[b] * row_v4;
+  uint4* dst = cache + plane * cache_plane_v4 + b * cache_seq_v4 + (size_t)sd.F[b] * row_v4;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = src[i];
+  if (blockIdx.x == 0 && plane == 0) {
+    const int L = sd.Lc[b];
+    const int ho = sd.head_off[b];
+    int32_t* t = tokens + (size_t)b * tok_stride + sd.Fp[b];
+    for (int i = threadIdx.x; i < L; i += blockDim.x) t[i] = yhat[ho + i];
+  }
+}
+
+__global__ void k_fill_mask(int32_t* tokens, int tok_stride, const int* __restrict__ P, const int* __restrict__ G,
+                            int mask_id) {
+  const int b = blockIdx.x;
+  for (int i = threadIdx.x; i < G[b]; i += blockDim.x) tokens[(size_t)b * tok_stride + P[b] + i] = mask_id;
+}
+
+// Rotary table in double precision: cs[pos][i] = (cos, sin)(pos * theta^(-2i/dh)), stored fp32.
+__global__ void k_rope_table(float2* __restrict__ cs, int max_len, int half, double theta) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= max_len * half) return;
+  const int pos = idx / half, i = idx % half;
+  const double inv = pow(theta, -(double)i / (double)half);
+  double s, c;
+  sincos((double)pos * inv, &s, &c);
+  cs[idx] = make_float2((float)c, (float)s);
+}
+
+}  // namespace lsp

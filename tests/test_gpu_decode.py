@@ -1,0 +1,167 @@
+"""End-to-end parity of the decode loop (Algorithm 1) against the oracle: per-step scores, boundaries,
+committed tokens, the KV cache contents, and the invariants on device state."""
+import numpy as np
+import pytest
+import torch
+
+import lsp_synth as S
+from oracle import scan as oscan
+from oracle.decode import decode, make_is_delim
+from gpu_util import DEV, make_pair, oracle_policy, tol_for
+
+pytestmark = pytest.mark.gpu
+NEAR = oscan.FLAG_NEAR_THRESHOLD | oscan.FLAG_NEAR_TIE
+
+
+def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, max_steps=None):
+    """Runs the GPU path step by step, committing the ORACLE's lengths, and compares every step's outputs."""
+    from paper_2603_05454_b200 import LSPDecoder
+    tol = tol_for(shape.dtype)
+    w_gpu, om = make_pair(shape, seed)
+    prompt = S.make_prompt(1, P, shape, seed)
+    sched.delim_bitmap = S.delimiter_bitmap(shape.vocab, *delim).to(DEV)
+    sched.flag_tol = tol
+    otok, orecs, (ock, ocv) = decode(om, prompt[0].numpy(), G, make_is_delim(*delim), oracle_policy(sched, tol),
+                                     score="pmax" if sched.score == 0 else "margin", max_steps=max_steps)
+    dec = LSPDecoder(shape, w_gpu, sched, 1, P + G, device=DEV)
+    if impl is not None:
+        dec.set_option(0, impl)
+    if attn_impl is not None:
+        dec.set_option(1, attn_impl)
+    tokens = torch.zeros(1, P + G, dtype=torch.int32, device=DEV)
+    tokens[0, :P] = prompt[0].to(DEV)
+    dec.begin(tokens, [P], [G])
+    n_flagged = 0
+    snap_prefix = None
+    for o in orecs:
+        rec = dec.denoise_step()[0]
+        y, p, m = dec.scores()
+        assert rec["n_before"] == o["n_before"] and rec["rows"] == o["rows"]
+        assert np.abs(p - o["pmax"]).max() <= tol, (o["step"], np.abs(p - o["pmax"]).max())
+        assert np.abs(m - o["delta"]).max() <= tol * max(1.0, 0.02 * np.abs(o["delta"]).max()), \
+            (o["step"], np.abs(m - o["delta"]).max())
+        diff = np.nonzero(y != o["yhat"])[0]
+        assert all(o["delta"][i] <= tol for i in diff), "argmax differs away from a near-tie"
+        if o["flags"] & NEAR or len(diff):
+            n_flagged += 1
+        else:
+            assert (rec["L_run"], rec["L_commit"]) == (o["L_run"], o["L_commit"]), (o["step"], rec)
+            assert rec["flags"] & ~NEAR == o["flags"] & ~NEAR
+        # prefix immutability on the device: tokens before the boundary never change
+        tk = tokens[0].cpu().numpy()
+        if snap_prefix is not None:
+            assert np.array_equal(tk[:len(snap_prefix)], snap_prefix)
+        dec.commit([o["L_commit"]])
+        # keep the device trajectory on the oracle's tokens even at a flagged near-tie
+        Fp = o["Fp"]
+        tokens[0, Fp:Fp + o["L_commit"]] = torch.tensor(o["yhat"][:o["L_commit"]], dtype=torch.int32, device=DEV)
+        torch.cuda.synchronize()
+        snap_prefix = tokens[0, :Fp + o["L_commit"]].cpu().numpy().copy()
+    if max_steps is None:
+        assert dec.active()[1] == 0
+        assert np.array_equal(tokens[0].cpu().numpy(), otok)
+    # cache contents: rows [0, F) equal the oracle's cache (same rounding points)
+    kv = dec.kv_view().float().cpu().numpy()
+    F = ock[0].shape[0]
+    for l in range(shape.n_layers):
+        kt = 4 * tol if shape.dtype == "bf16" else tol
+        np.testing.assert_allclose(kv[l, 0, 0, :F], ock[l], atol=kt * max(1.0, np.abs(ock[l]).max()))
+        np.testing.assert_allclose(kv[l, 1, 0, :F], ocv[l], atol=kt * max(1.0, np.abs(ocv[l]).max()))
+    assert not kv[:, :, 0, F:].any()          # nothing beyond the committed prefix was ever written
+    dec.close()
+    return len(orecs), n_flagged
+
+
+def test_cfg1_fp32_full_decode_as_written():
+    from paper_2603_05454_b200 import SchedCfg
+    w = S.config("cfg1")
+    steps, flagged = _teacher_forced(w.shape, 0, w.prompt_len, w.gen_len, SchedCfg(tau=w.tau), w.delim)
+    assert steps >= 1
+
+
+def test_cfg1_fp32_margin_score_and_lower_threshold_multi_token_commits():
+    from paper_2603_05454_b200 import SchedCfg
+    w = S.config("cfg1")
+    # the configuration as written commits one token per step (max-prob stays near 0.12); a threshold inside
+    # the observed score range exercises multi-token runs on the same model
+    steps, _ = _teacher_forced(w.shape, 0, w.prompt_len, w.gen_len, SchedCfg(tau=0.1205), w.delim)
+    assert steps < w.gen_len
+    _teacher_forced(w.shape, 0, w.prompt_len, w.gen_len, SchedCfg(score=1, tau=0.945), (1, 400))
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("hkv", [4, 2, 1])
+def test_small_models_mha_gqa(dtype, hkv):
+    from paper_2603_05454_b200 import SchedCfg
+    sh = S.ModelShape(2, 256, 4, hkv, 64, 512, 1024, dtype=dtype, head_scale=1.5, w_std=0.0625)
+    _teacher_forced(sh, 3, 24, 40, SchedCfg(tau=0.05), (1, 200))
+    _teacher_forced(sh, 4, 24, 40, SchedCfg(mode=1, alpha=0.25, beta=0.5), (1, 200))
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+def test_bf16_head_dim_128_model(impl):
+    from paper_2603_05454_b200 import SchedCfg
+    sh = S.ModelShape(2, 512, 4, 2, 128, 1024, 4096, dtype="bf16", head_scale=1.5, w_std=0.044)
+    _teacher_forced(sh, 5, 40, 90, SchedCfg(tau=0.04), (1, 400), impl=impl)
+
+
+def test_batched_ragged_free_running_matches_per_sequence_oracle():
+    """Sequences of a batch are independent: a ragged batch must reproduce each sequence's own oracle decode
+    (free-running; a step flagged near a threshold or tie ends the comparison for that sequence)."""
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+    sh = S.ModelShape(2, 256, 4, 2, 64, 512, 1024, dtype="fp32", head_scale=1.5, w_std=0.0625)
+    w_gpu, om = make_pair(sh, 9)
+    Ps, Gs = [5, 17, 32], [30, 9, 64]
+    B, stride = 3, 96
+    sched = SchedCfg(tau=0.05, delim_bitmap=S.delimiter_bitmap(sh.vocab, 1, 200).to(DEV), flag_tol=1e-4)
+    prompts = S.make_prompt(B, 32, sh, 11)
+    tokens = torch.zeros(B, stride, dtype=torch.int32, device=DEV)
+    for b in range(B):
+        tokens[b, :Ps[b]] = prompts[b, :Ps[b]].to(DEV)
+    dec = LSPDecoder(sh, w_gpu, sched, B, stride, device=DEV)
+    dec.begin(tokens, Ps, Gs)
+    n_steps, recs = dec.generate(max_recs=B * 200)
+    torch.cuda.synchronize()
+    tk = tokens.cpu().numpy()
+    for b in range(B):
+        otok, orecs, _ = decode(om, prompts[b, :Ps[b]].numpy(), Gs[b], make_is_delim(1, 200),
+                                oracle_policy(sched, 1e-4))
+        mine = [r for i, r in enumerate(recs) if i % B == b and r["n_before"] > 0]
+        ok = True
+        for r, o in zip(mine, orecs):
+            if o["flags"] & NEAR:
+                ok = False
+                break
+            assert (r["L_run"], r["L_commit"], r["n_before"]) == (o["L_run"], o["L_commit"], o["n_before"])
+        if ok:
+            assert len(mine) == len(orecs)
+            assert np.array_equal(tk[b, :Ps[b] + Gs[b]], otok)
+        assert (tk[b, :Ps[b] + Gs[b]] != sh.mask_id).all()
+    dec.close()
+
+
+def test_state_errors_leave_state_unchanged():
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg, LSPError
+    sh = S.ModelShape(1, 64, 1, 1, 64, 64, 256, dtype="fp32")
+    dec = LSPDecoder(sh, S.make_weights(sh, 0, device=DEV), SchedCfg(tau=2.0), 1, 16, device=DEV)
+    tokens = torch.zeros(1, 16, dtype=torch.int32, device=DEV)
+    with pytest.raises(LSPError):
+        dec.batch = 1
+        dec.denoise_step()                      # before begin
+    dec.begin(tokens, [4], [3])
+    with pytest.raises(LSPError) as e:
+        dec.commit()                            # no step yet
+    assert e.value.code == -4
+    dec.denoise_step()
+    for bad in (0, 4, -1):
+        with pytest.raises(LSPError):
+            dec.commit([bad])
+    assert dec.active()[0][0] == 3
+    dec.commit([1])
+    with pytest.raises(LSPError):
+        dec.commit([1])                         # needs a new step
+    n, _ = dec.generate()
+    assert n == 2 and dec.active()[1] == 0
+    with pytest.raises(LSPError):
+        dec.denoise_step()                      # already finished
+    dec.close()

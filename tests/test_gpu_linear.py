@@ -1,0 +1,55 @@
+"""K3 parity: the GEMM kernels with their fused epilogues against fp64 matrix products."""
+import numpy as np
+import pytest
+import torch
+
+import lsp_synth as S
+from oracle import dlm
+from gpu_util import DEV
+
+pytestmark = pytest.mark.gpu
+
+
+def _dec(dtype):
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+    sh = S.ModelShape(1, 64, 1, 1, 64, 64, 128, dtype=dtype)
+    return LSPDecoder(sh, S.make_weights(sh, 0, device=DEV), SchedCfg(), 1, 8, device=DEV)
+
+
+def _check(dtype, impl, M, N, K, seed):
+    tdt = torch.float32 if dtype == "fp32" else torch.bfloat16
+    dec = _dec(dtype)
+    dec.set_option(0, impl)
+    A = S.normal((M, K), seed, 1, 1.0, tdt, DEV)
+    W = S.normal((N, K), seed, 2, 0.05, tdt, DEV)
+    W2 = S.normal((N, K), seed, 3, 0.05, tdt, DEV)
+    X0 = S.normal((M, N), seed, 4, 1.0, tdt, DEV)
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    rnd = dlm.round_bf16 if dtype == "bf16" else (lambda x: x.astype(np.float32).astype(np.float64))
+    a, w, w2, x0 = f64(A), f64(W), f64(W2), f64(X0)
+    rtol = 2e-5 if dtype == "fp32" else 1.0 / 128   # one bf16 ulp of the result (rounding point may flip)
+    out = torch.empty(M, N, dtype=tdt, device=DEV)
+    dec.op_linear(0, A, W, None, out)
+    ref = a @ w.T
+    np.testing.assert_allclose(f64(out), rnd(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05)
+    xr = X0.clone()
+    dec.op_linear(1, A, W, None, xr)
+    ref = x0 + a @ w.T
+    np.testing.assert_allclose(f64(xr), rnd(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05)
+    dec.op_linear(2, A, W, W2, out)
+    g, u = a @ w.T, a @ w2.T
+    ref = g / (1 + np.exp(-g)) * u
+    np.testing.assert_allclose(f64(out), rnd(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05)
+    dec.close()
+
+
+@pytest.mark.parametrize("shape", [(1, 64, 64), (70, 136, 192), (129, 256, 128), (300, 512, 1024)])
+def test_linear_fp32(shape):
+    _check("fp32", 0, *shape, seed=0)
+
+
+@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("shape", [(1, 64, 64), (70, 136, 192), (129, 256, 128), (300, 512, 1024),
+                                   (512, 4096, 4096), (37, 12288, 4096), (257, 4096, 12288)])
+def test_linear_bf16(impl, shape):
+    _check("bf16", impl, *shape, seed=1)
