@@ -70,7 +70,8 @@ typedef struct {
   int fixed_k;
   const uint8_t* delim_bitmap; /* device, (vocab+7)/8 bytes, bit (v & 7) of byte v >> 3; NULL = empty set D */
   int exclude_mask_logit;      /* 1: the mask_id column takes no part in argmax / margin / probability */
-  float flag_tol;              /* tolerance of the NEAR_THRESHOLD / NEAR_TIE flags; 0 disables them */
+  float flag_tol;              /* NEAR_THRESHOLD flag: |score_i - tau| <= flag_tol for some i <= L'+1; 0 disables */
+  float tie_tol;               /* NEAR_TIE flag: delta_i <= tie_tol for some committed i; 0 disables */
 } lsp_sched_cfg;
 
 /* Device pointers to the weights, all element type T.  Per-layer arrays are HOST arrays of

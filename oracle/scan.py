@@ -82,7 +82,7 @@ def snap_to_delimiter(yhat, L_run, N, is_delim, l_min, W):
 
 
 def lsp_scan(score, yhat, is_delim, mode=MODE_FIXED_TAU, tau=0.9, alpha=0.25, beta=0.5,
-             l_min=1, W=16, fixed_k=1, flag_tol=0.0, margin=None):
+             l_min=1, W=16, fixed_k=1, flag_tol=0.0, tie_tol=0.0, margin=None):
     """One scheduler decision for one sequence.  Returns a dict with L_run (L'), L_commit (L),
     tau_used and flags."""
     N = len(score)
@@ -105,8 +105,8 @@ def lsp_scan(score, yhat, is_delim, mode=MODE_FIXED_TAU, tau=0.9, alpha=0.25, be
         for i in range(min(N, L_run + 1)):
             if abs(float(score[i]) - tau_used) <= flag_tol:
                 flags |= FLAG_NEAR_THRESHOLD
-        if margin is not None:
-            for i in range(L):
-                if float(margin[i]) <= flag_tol:
-                    flags |= FLAG_NEAR_TIE
+    if tie_tol > 0 and margin is not None:
+        for i in range(L):
+            if float(margin[i]) <= tie_tol:
+                flags |= FLAG_NEAR_TIE
     return dict(L_run=L_run, L_commit=L, tau_used=tau_used, flags=flags)

@@ -35,7 +35,7 @@ class ModelCfg(C.Structure):
 class SchedCfgC(C.Structure):
     _fields_ = [("score", C.c_int), ("mode", C.c_int), ("tau", C.c_float), ("alpha", C.c_float), ("beta", C.c_float),
                 ("l_min", C.c_int), ("snap_window", C.c_int), ("fixed_k", C.c_int), ("delim_bitmap", C.c_void_p),
-                ("exclude_mask_logit", C.c_int), ("flag_tol", C.c_float)]
+                ("exclude_mask_logit", C.c_int), ("flag_tol", C.c_float), ("tie_tol", C.c_float)]
 
 
 class WeightsC(C.Structure):
@@ -94,11 +94,12 @@ class SchedCfg:
     delim_bitmap: Optional[torch.Tensor] = None   # uint8 CUDA tensor, vocab bits
     exclude_mask_logit: int = 1
     flag_tol: float = 0.0
+    tie_tol: float = 0.0
 
     def to_c(self) -> SchedCfgC:
         p = self.delim_bitmap.data_ptr() if self.delim_bitmap is not None else None
         return SchedCfgC(self.score, self.mode, self.tau, self.alpha, self.beta, self.l_min, self.snap_window,
-                         self.fixed_k, p, self.exclude_mask_logit, self.flag_tol)
+                         self.fixed_k, p, self.exclude_mask_logit, self.flag_tol, self.tie_tol)
 
 
 def _ptr_array(tensors: Sequence[torch.Tensor]):

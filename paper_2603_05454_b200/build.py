@@ -8,7 +8,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblsp_b200.so")
 SOURCES = ["lsp_api.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-shared", "--expt-relaxed-constexpr", "-DLSP_NO_UMMA"]
+              "-Xcompiler", "-fPIC", "-shared", "--expt-relaxed-constexpr"]
 
 
 def _newest_source_mtime():

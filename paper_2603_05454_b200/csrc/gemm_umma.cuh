@@ -1,0 +1,484 @@
+// bf16 GEMM on the 5th-generation tensor cores (tcgen05) for sm_100a.
+//
+//   acc[m, c] = sum_k A[m, k] * Wt[c, k]        A: [M, K] bf16 row-major, Wt: weight rows, K-major, fp32 accumulate
+//
+// One CTA computes a 128 x BN accumulator tile that lives in tensor memory (TMEM).  Operand tiles are brought
+// into 128-byte-swizzled shared memory by TMA (cp.async.bulk.tensor, no multicast) through a ring of stages
+// guarded by mbarriers; a single thread issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction) and
+// releases each stage with tcgen05.commit; four epilogue warps read the accumulators back with tcgen05.ld
+// (each thread owns one output row) and run the fused epilogue (store / residual / SwiGLU / rotary+KV staging /
+// LM-head top-2 + log-sum-exp reduction).
+//
+// The B tile is two TMA boxes of BN/2 weight rows each (possibly from two tensors), so accumulator columns
+// c and c + BN/2 of one thread hold the pair an element-wise fusion needs (gate/up, rotate-half partners).
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = epilogue.
+// Every wait is bounded by wall-clock time; on expiry the kernel records (code, site) in a status word, lets
+// all roles drain and returns, so a protocol error can never hang the device.
+#pragma once
+#include <cuda.h>
+
+#include <map>
+#include <string>
+#include <tuple>
+
+#include "epilogues.cuh"
+
+namespace lsp {
+
+constexpr int UM_BM = 128;
+constexpr int UM_BK = 64;                 // bf16 elements = one 128-byte swizzle row
+constexpr int UM_THREADS = 192;
+constexpr int UM_MAX_STAGES = 12;
+constexpr uint64_t UM_WAIT_NS = 2000000000ull;   // 2 s
+
+// ---- PTX wrappers -----------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait.  Returns false after UM_WAIT_NS or when another role has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  uint64_t t0 = 0;
+  for (uint32_t spin = 0;; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spin & 1023u) == 1023u) {
+      if (*abort_flag) return false;
+      const uint64_t now = globaltimer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > UM_WAIT_NS) return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor for a K-major bf16 tile stored as rows of 128 bytes with the 128-byte swizzle:
+// 8-row groups are 1024 bytes apart (stride byte offset); the leading byte offset is unused for this layout.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                          // leading byte offset (ignored with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset
+  d |= (uint64_t)1 << 46;                          // descriptor version for this architecture
+  d |= (uint64_t)2 << 61;                          // layout: 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t make_idesc(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(UM_BM >> 4) << 24);
+}
+
+// ---- vector helpers for the epilogues ------------------------------------------------------------------
+__device__ __forceinline__ uint4 pack8(const float* v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
+  __nv_bfloat162 b = __floats2bfloat162_rn(v[2], v[3]);
+  __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]);
+  __nv_bfloat162 d = __floats2bfloat162_rn(v[6], v[7]);
+  uint4 r;
+  r.x = *reinterpret_cast<uint32_t*>(&a);
+  r.y = *reinterpret_cast<uint32_t*>(&b);
+  r.z = *reinterpret_cast<uint32_t*>(&c);
+  r.w = *reinterpret_cast<uint32_t*>(&d);
+  return r;
+}
+__device__ __forceinline__ void unpack8(const uint4& u, float* v) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __low2float(p[i]);
+    v[2 * i + 1] = __high2float(p[i]);
+  }
+}
+
+// 16 consecutive pair indices j..j+15 of row m (a1 unused for plain epilogues).
+__device__ __forceinline__ void epi16(const EpiStore<bf16>& e, int m, int j, const float* a0, const float*) {
+  uint4* p = reinterpret_cast<uint4*>(e.out + (size_t)m * e.ld + j);
+  p[0] = pack8(a0);
+  p[1] = pack8(a0 + 8);
+}
+__device__ __forceinline__ void epi16(const EpiResidual<bf16>& e, int m, int j, const float* a0, const float*) {
+  uint4* p = reinterpret_cast<uint4*>(e.x + (size_t)m * e.ld + j);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float x[8];
+    unpack8(p[h], x);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] += a0[8 * h + i];
+    p[h] = pack8(x);
+  }
+}
+__device__ __forceinline__ void epi16(const EpiSwiGLU<bf16>& e, int m, int j, const float* g, const float* u) {
+  float r[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) r[i] = g[i] / (1.f + __expf(-g[i])) * u[i];
+  uint4* p = reinterpret_cast<uint4*>(e.out + (size_t)m * e.ld + j);
+  p[0] = pack8(r);
+  p[1] = pack8(r + 8);
+}
+__device__ __forceinline__ void epi16(const EpiQKVRope<bf16>& e, int m, int j, const float* a0, const float* a1) {
+  const int h = j / e.half, i = j % e.half;       // 16 indices stay inside one head (half is a multiple of 16)
+  const int dh = 2 * e.half;
+  float r0[16], r1[16];
+  bf16* dst;
+  if (h < e.n_heads + e.n_kv_heads) {
+    const float4* c4 = reinterpret_cast<const float4*>(e.cs + (size_t)e.row_pos[m] * e.half + i);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float4 c = __ldg(c4 + q);             // (cos, sin) of two consecutive frequencies
+      r0[2 * q] = a0[2 * q] * c.x - a1[2 * q] * c.y;
+      r1[2 * q] = a1[2 * q] * c.x + a0[2 * q] * c.y;
+      r0[2 * q + 1] = a0[2 * q + 1] * c.z - a1[2 * q + 1] * c.w;
+      r1[2 * q + 1] = a1[2 * q + 1] * c.z + a0[2 * q + 1] * c.w;
+    }
+    dst = (h < e.n_heads) ? e.q_out + (size_t)m * e.n_heads * dh + h * dh
+                          : e.k_stage + (size_t)m * e.n_kv_heads * dh + (h - e.n_heads) * dh;
+  } else {
+#pragma unroll
+    for (int q = 0; q < 16; ++q) { r0[q] = a0[q]; r1[q] = a1[q]; }
+    dst = e.v_stage + (size_t)m * e.n_kv_heads * dh + (h - e.n_heads - e.n_kv_heads) * dh;
+  }
+  uint4* p0 = reinterpret_cast<uint4*>(dst + i);
+  uint4* p1 = reinterpret_cast<uint4*>(dst + i + e.half);
+  p0[0] = pack8(r0);
+  p0[1] = pack8(r0 + 8);
+  p1[0] = pack8(r1);
+  p1[1] = pack8(r1 + 8);
+}
+
+// ---- the kernel -------------------------------------------------------------------------------------------
+struct UmmaArgs {
+  int M;        // activation rows
+  int n_pairs;  // dual: pair indices (each tile covers BN/2); plain: output columns (each tile covers BN)
+  int K;
+  int num_kb;   // K / 64
+  int stages;
+  int m_fast;   // 1: blockIdx.x walks the row tiles (keeps one weight tile hot in L2 across the rows), 0: the column tiles
+  unsigned* status;
+};
+
+template <int BN>
+constexpr int umma_stage_bytes() { return UM_BM * UM_BK * 2 + BN * UM_BK * 2; }
+
+template <int BN, typename Epi>
+__global__ void __launch_bounds__(UM_THREADS, 1)
+k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
+            const __grid_constant__ CUtensorMap map_b1, UmmaArgs args, Epi epi) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int A_BYTES = UM_BM * UM_BK * 2;
+  constexpr int B_HALF_BYTES = (BN / 2) * UM_BK * 2;
+  constexpr int STAGE_BYTES = A_BYTES + 2 * B_HALF_BYTES;
+  constexpr int HALF = BN / 2;
+  // 1024-byte alignment for the swizzled tiles
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int S = args.stages;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * STAGE_BYTES);
+  // bars[0..S) = full, bars[S..2S) = empty, bars[2S] = accumulator ready
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 1);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = (args.m_fast ? blockIdx.x : blockIdx.y) * UM_BM;
+  const int tile = args.m_fast ? blockIdx.y : blockIdx.x;
+  // weight rows of the two boxes
+  int row_b0, row_b1;
+  if (Epi::kDual) {
+    row_b0 = epi.row0(tile * HALF);
+    row_b1 = epi.row1(tile * HALF);
+  } else {
+    row_b0 = tile * BN;
+    row_b1 = tile * BN + HALF;
+  }
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+  const uint32_t acc_bar = bar_base + 8u * (2 * S);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(acc_bar, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)BN)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int num_kb = args.num_kb;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
+        const int s = kb % S;
+        const uint32_t ph = (uint32_t)(kb / S) & 1u;
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
+          if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 1u; }
+          ok = false;
+          break;
+        }
+        mbar_expect_tx(full_bar(s), STAGE_BYTES);
+        const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
+        tma_load_2d(sa, &map_a, kb * UM_BK, m0, full_bar(s));
+        tma_load_2d(sa + A_BYTES, &map_b0, kb * UM_BK, row_b0, full_bar(s));
+        tma_load_2d(sa + A_BYTES + B_HALF_BYTES, &map_b1, kb * UM_BK, row_b1, full_bar(s));
+        ++issued;
+      }
+      // Do not leave while copies may still be landing in this CTA's shared memory.
+      const int first = issued > S ? issued - S : 0;
+      for (int kb = first; kb < issued; ++kb) {
+        volatile uint32_t no_abort = 0;
+        mbar_wait(full_bar(kb % S), (uint32_t)(kb / S) & 1u, &no_abort);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(BN);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % S;
+        const uint32_t ph = (uint32_t)(kb / S) & 1u;
+        if (!mbar_wait(full_bar(s), ph, abort_flag)) {
+          if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 2u; }
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
+        const uint64_t da = make_smem_desc(sa);
+        const uint64_t db = make_smem_desc(sa + A_BYTES);
+#pragma unroll
+        for (int k = 0; k < UM_BK / 16; ++k) {
+          // advance 16 bf16 = 32 bytes = 2 descriptor units along K inside the swizzle row
+          tc_mma_f16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+        }
+        tc_commit(empty_bar(s));     // frees the stage once these MMAs have read it
+      }
+      if (ok) tc_commit(acc_bar);    // accumulator complete
+    }
+  } else {
+    // ---------------- epilogue (warps 2..5) ----------------
+    const int q = warp & 3;                        // TMEM lane quarter this warp may access
+    const int m = m0 + q * 32 + lane;
+    bool ok = mbar_wait(acc_bar, 0u, abort_flag);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) {
+      if (lane == 0 && !*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 3u; }
+    } else {
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+      if constexpr (Epi::kReduce) {
+        Top2 r = top2_empty();
+        const int col0 = tile * BN;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 16) {
+          float v[16];
+          tc_ld16(t_row + c, v);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int col = col0 + c + i;
+            if (epi.valid(col)) top2_push(r, v[i], col);
+          }
+        }
+        if (m < args.M) epi.part[(size_t)m * epi.n_tiles + tile] = r;
+      } else if constexpr (Epi::kDual) {
+        const int j0 = tile * HALF;
+#pragma unroll 1
+        for (int c = 0; c < HALF; c += 16) {
+          float a0[16], a1[16];
+          tc_ld16(t_row + c, a0);
+          tc_ld16(t_row + HALF + c, a1);
+          if (m < args.M && j0 + c < args.n_pairs) epi16(epi, m, j0 + c, a0, a1);
+        }
+      } else {
+        const int j0 = tile * BN;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 16) {
+          float a0[16];
+          tc_ld16(t_row + c, a0);
+          if (m < args.M && j0 + c < args.n_pairs) epi16(epi, m, j0 + c, a0, a0);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)BN) : "memory");
+  }
+}
+
+// ---- host side ------------------------------------------------------------------------------------------------
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct UmmaState {
+  PFN_encodeTiled encode = nullptr;
+  std::map<std::tuple<const void*, int, int, int>, CUtensorMap> cache;
+  int max_smem = 0;
+  std::string err;
+};
+
+inline int umma_init(UmmaState& st) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess) {
+    st.err = "cuTensorMapEncodeTiled not available";
+    return -1;
+  }
+  st.encode = (PFN_encodeTiled)fn;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&st.max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  return 0;
+}
+
+// 2-D bf16 tensor [rows, K] row-major, box = [64 (K), box_rows], 128-byte swizzle, zero fill out of bounds.
+inline const CUtensorMap* umma_map(UmmaState& st, const void* base, int rows, int K, int box_rows) {
+  auto key = std::make_tuple(base, rows, K, box_rows);
+  auto it = st.cache.find(key);
+  if (it != st.cache.end()) return &it->second;
+  CUtensorMap m;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)UM_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = st.encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    st.err = "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")";
+    return nullptr;
+  }
+  return &st.cache.emplace(key, m).first->second;
+}
+
+constexpr int UM_HEAD_BN = 256;
+inline int umma_head_tiles(int vocab) { return (vocab + UM_HEAD_BN - 1) / UM_HEAD_BN; }
+
+template <int BN, typename Epi>
+int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
+                int n_rows_w, const Epi& epi, unsigned* status) {
+  constexpr int stage = umma_stage_bytes<BN>();
+  const int aux = 1024 /*alignment slack*/ + 8 * (2 * UM_MAX_STAGES + 1) + 16;
+  int stages = (st.max_smem - aux) / stage;
+  if (stages > UM_MAX_STAGES) stages = UM_MAX_STAGES;
+  const int num_kb = K / UM_BK;
+  if (stages > num_kb) stages = num_kb;
+  if (stages < 1) { st.err = "not enough shared memory"; return -2; }
+  const size_t smem = (size_t)stages * stage + aux;
+  static bool attr_set = false;   // per instantiation
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_umma<BN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, st.max_smem);
+    if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -3; }
+    attr_set = true;
+  }
+  if (st.cache.size() > 4096) st.cache.clear();
+  const CUtensorMap* ma = umma_map(st, A, M, K, UM_BM);
+  const CUtensorMap* mb0 = umma_map(st, W0, n_rows_w, K, BN / 2);
+  const CUtensorMap* mb1 = umma_map(st, W1, n_rows_w, K, BN / 2);
+  if (!ma || !mb0 || !mb1) return -4;
+  const int per_tile = Epi::kDual ? BN / 2 : BN;
+  const int m_fast = Epi::kReduce ? 1 : 0;
+  dim3 grid((NP + per_tile - 1) / per_tile, (M + UM_BM - 1) / UM_BM);
+  if (m_fast) grid = dim3(grid.y, grid.x);
+  UmmaArgs args{M, NP, K, num_kb, stages, m_fast, status};
+  k_gemm_umma<BN, Epi><<<grid, UM_THREADS, smem, stream>>>(*ma, *mb0, *mb1, args, epi);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
+  return 0;
+}
+
+// Tile-width choice: the widest tile that still gives every SM a CTA; the rotary epilogue needs both partners of a
+// pair inside one head, which caps the tile at head_dim columns.
+template <typename Epi>
+int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
+              int n_rows_w, const Epi& epi, unsigned* status) {
+  if (K % UM_BK) { st.err = "K must be a multiple of 64"; return -6; }
+  if constexpr (Epi::kReduce) {
+    return umma_launch<UM_HEAD_BN, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+  } else {
+    const int cols = Epi::kDual ? 2 * NP : NP;
+    const int mt = (M + UM_BM - 1) / UM_BM;
+    int max_bn = 256;
+    if constexpr (std::is_same<Epi, EpiQKVRope<bf16>>::value) max_bn = 2 * epi.half;
+    int bn = 32;
+    for (int cand = 256; cand >= 32; cand >>= 1) {
+      if (cand > max_bn) continue;
+      if ((long)mt * ((cols + cand - 1) / cand) >= 148) { bn = cand; break; }
+    }
+    switch (bn) {
+      case 256: return umma_launch<256, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+      case 128: return umma_launch<128, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+      case 64: return umma_launch<64, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+      default: return umma_launch<32, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+    }
+  }
+}
+
+}  // namespace lsp

@@ -195,6 +195,7 @@ ScanParams scan_params(const lsp_ctx* c) {
   p.fixed_k = c->s.fixed_k;
   p.delim = c->s.delim_bitmap;
   p.flag_tol = c->s.flag_tol;
+  p.tie_tol = c->s.tie_tol;
   return p;
 }
 
@@ -658,7 +659,7 @@ int lsp_scan(lsp_ctx* c, const float* score, const int32_t* yhat, const float* m
 int lsp_op_linear(lsp_ctx* c, int op, const void* A, const void* W, const void* W2, void* out, int M, int N, int K) {
   if (!c || !A || !W || !out || M < 0 || N < 1 || K < 1) return LSP_ERR_ARG;
   if (op < 0 || op > 2 || (op == 2 && !W2)) return fail(c, LSP_ERR_ARG, "lsp_op_linear: bad op");
-  if (K % 64 || N % 8) return fail(c, LSP_ERR_SHAPE, "lsp_op_linear: K must be a multiple of 64 and N of 8");
+  if (K % 64 || N % 16) return fail(c, LSP_ERR_SHAPE, "lsp_op_linear: K must be a multiple of 64 and N of 16");
   const int rc = c->m.dtype == 0 ? op_linear_impl<float>(c, op, A, W, W2, out, M, N, K)
                                  : op_linear_impl<bf16>(c, op, A, W, W2, out, M, N, K);
   if (rc) return rc;

@@ -92,7 +92,7 @@ struct ScanParams {
   float tau, alpha, beta;
   int l_min, W, fixed_k;
   const uint8_t* delim;
-  float flag_tol;
+  float flag_tol, tie_tol;
 };
 
 __device__ __forceinline__ bool is_delim(const uint8_t* bm, int id) {
@@ -181,12 +181,13 @@ __global__ void k_lsp_scan(const float* __restrict__ score, const int32_t* __res
     if (Lrun < max(1, p.l_min)) flags |= 2u;
   }
   L = min(N, max(L, 1));
-  if (p.flag_tol > 0.f) {
+  if (p.flag_tol > 0.f || p.tie_tol > 0.f) {
     bool near = false, tie = false;
     const int lim = min(N, Lrun + 1);
-    for (int i = lane; i < lim; i += 32) near |= fabsf(sc[i] - tau) <= p.flag_tol;
-    if (margin != nullptr)
-      for (int i = lane; i < L; i += 32) tie |= margin[base + i] <= p.flag_tol;
+    if (p.flag_tol > 0.f)
+      for (int i = lane; i < lim; i += 32) near |= fabsf(sc[i] - tau) <= p.flag_tol;
+    if (margin != nullptr && p.tie_tol > 0.f)
+      for (int i = lane; i < L; i += 32) tie |= margin[base + i] <= p.tie_tol;
     if (__any_sync(0xffffffffu, near)) flags |= 16u;
     if (__any_sync(0xffffffffu, tie)) flags |= 32u;
   }

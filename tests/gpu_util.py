@@ -10,7 +10,18 @@ DEV = "cuda:0"
 
 
 def tol_for(dtype):
+    """Tolerance on probabilities (and on logits of unit scale)."""
     return 1e-4 if dtype == "fp32" else 2e-2
+
+
+def tol_logit(dtype, z_rms):
+    """Tolerance on logit-scale quantities (logits, the margin delta).  fp32: 1e-4 relative to the logit scale.
+    bf16: two correct bf16 pipelines agree to about one bf16 ulp (2^-8 relative) per element at every rounding
+    point, which reaches the logits as noise of roughly 2^-8 * z_rms per rounding stage; 2^-5 * z_rms bounds the
+    maximum over a few thousand (row, column) pairs and a handful of stages, with 2e-2 as the floor."""
+    if dtype == "fp32":
+        return 1e-4 * max(1.0, z_rms)
+    return max(2e-2, z_rms / 32.0)
 
 
 def make_pair(shape, seed):
@@ -20,7 +31,8 @@ def make_pair(shape, seed):
     return w_gpu, dlm.OracleDLM(shape, w_cpu)
 
 
-def oracle_policy(s, flag_tol):
+def oracle_policy(s, flag_tol=None):
     """kwargs of oracle.scan.lsp_scan that mirror a binding SchedCfg (thresholds as the fp32 values the GPU sees)."""
     return dict(mode=s.mode, tau=float(np.float32(s.tau)), alpha=float(np.float32(s.alpha)),
-                beta=float(np.float32(s.beta)), l_min=s.l_min, W=s.snap_window, fixed_k=s.fixed_k, flag_tol=flag_tol)
+                beta=float(np.float32(s.beta)), l_min=s.l_min, W=s.snap_window, fixed_k=s.fixed_k,
+                flag_tol=float(np.float32(s.flag_tol)), tie_tol=float(np.float32(s.tie_tol)))

@@ -6,7 +6,7 @@ import torch
 import lsp_synth as S
 from oracle import scan as oscan
 from oracle.scores import scores_from_logits
-from gpu_util import DEV, tol_for
+from gpu_util import DEV, tol_for, tol_logit
 
 pytestmark = pytest.mark.gpu
 
@@ -24,30 +24,34 @@ def _run(dtype, d, V, lens, head_scale, tau, seed=0, exclude=1, impl=None):
     rows = int(sum(lens))
     bm = S.delimiter_bitmap(V, 1, 32).to(DEV)
     tol = tol_for(dtype)
-    sched = SchedCfg(tau=tau, delim_bitmap=bm, exclude_mask_logit=exclude, flag_tol=tol)
+    # oracle: full logits in fp64 from the same (dtype-rounded) values
+    hidden = S.normal((rows, d), seed, 77, 1.0, tdt, DEV)
+    h64 = hidden.float().cpu().numpy().astype(np.float64)
+    w64 = w["w_head"].float().cpu().numpy().astype(np.float64)
+    logits = h64 @ w64.T
+    # inputs are identical on both sides here, so only accumulation order differs: fp32 accumulation of d
+    # products of magnitude ~z_rms/sqrt(d) keeps logits within 1e-4 * z_rms even in bf16
+    tol_z = tol_logit("fp32", float(np.sqrt((logits * logits).mean())))
+    sched = SchedCfg(tau=tau, delim_bitmap=bm, exclude_mask_logit=exclude, flag_tol=tol, tie_tol=tol_z)
     dec = LSPDecoder(sh, w, sched, len(lens), max(2, max(lens)), device=DEV)
     if impl is not None:
         dec.set_option(0, impl)
-    hidden = S.normal((rows, d), seed, 77, 1.0, tdt, DEV)
     off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
     out = dec.head_scan(hidden, off)
     y, p, m = dec.scores()
     dec.close()
-    # oracle: full logits in fp64 from the same (dtype-rounded) values
-    h64 = hidden.float().cpu().numpy().astype(np.float64)
-    w64 = w["w_head"].float().cpu().numpy().astype(np.float64)
-    yo, po, mo = scores_from_logits(h64 @ w64.T, sh.mask_id if exclude else -1)
-    assert np.abs(p - po).max() <= tol
-    assert np.abs(m - mo).max() <= tol
+    yo, po, mo = scores_from_logits(logits, sh.mask_id if exclude else -1)
+    assert np.abs(p - po).max() <= 1e-4
+    assert np.abs(m - mo).max() <= tol_z
     bad = np.nonzero(y != yo)[0]
-    assert all(mo[i] <= tol for i in bad), "argmax differs away from a near-tie"
+    assert all(mo[i] <= tol_z for i in bad), "argmax differs away from a near-tie"
     n_flag = 0
     for b in range(len(lens)):
         a, e = off[b], off[b + 1]
         if e == a:
             continue
         r = oscan.lsp_scan(po[a:e], yo[a:e], lambda t: 1 <= t <= 32, tau=float(np.float32(tau)), W=16,
-                           flag_tol=tol, margin=mo[a:e])
+                           flag_tol=float(np.float32(tol)), tie_tol=float(np.float32(tol_z)), margin=mo[a:e])
         if r["flags"] & (oscan.FLAG_NEAR_THRESHOLD | oscan.FLAG_NEAR_TIE):
             n_flag += 1
             continue

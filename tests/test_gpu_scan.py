@@ -44,6 +44,7 @@ def _case(dec, lens, seed, sched, p_pass=0.8, dens=0.12):
                            tau=float(np.float32(sched.tau)), alpha=float(np.float32(sched.alpha)),
                            beta=float(np.float32(sched.beta)), l_min=sched.l_min, W=sched.snap_window,
                            fixed_k=sched.fixed_k, flag_tol=float(np.float32(sched.flag_tol)),
+                           tie_tol=float(np.float32(sched.tie_tol)),
                            margin=(scores[b] * 3).numpy())
         assert out["L_run"][b] == r["L_run"], (b, n, out["L_run"][b], r)
         assert out["L_commit"][b] == r["L_commit"], (b, n, out["L_commit"][b], r)
@@ -60,7 +61,7 @@ LENS = [1, 2, 31, 32, 33, 64, 65, 100, 255, 256, 257, 1024, 1000, 7, 0, 513]
 def test_fixed_tau(dec, W, l_min):
     from paper_2603_05454_b200 import SchedCfg
     for seed, pp in ((0, 0.8), (1, 0.97), (2, 0.3), (3, 1.0)):
-        _case(dec, LENS, seed, SchedCfg(tau=0.9, snap_window=W, l_min=l_min, flag_tol=0.01), p_pass=pp)
+        _case(dec, LENS, seed, SchedCfg(tau=0.9, snap_window=W, l_min=l_min, flag_tol=0.01, tie_tol=0.4), p_pass=pp)
 
 
 def test_adaptive_and_fixed_k(dec):
