@@ -120,7 +120,13 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
 int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
 
 /* Options: key 0 = GEMM implementation for bf16 (0 = CUDA-core reference kernels, 1 = tcgen05,
- * default 1); key 1 = attention implementation for bf16 (0 = CUDA-core, 1 = tensor-core). */
+ * default 1); key 1 = attention implementation for bf16 (0 = CUDA-core, 1 = tensor-core);
+ * key 2 = per-class CUDA-event timing (0 off, 1 on; see lsp_last_timing);
+ * key 3 = lsp_op_linear returns without synchronising or checking the device status (1) or not (0);
+ * key 4 = lsp_op_linear enqueues the operation this many times (timing aid); key 5 = repetition r reads its weights
+ * at W + (r mod value) * N * K elements, so a buffer of several weight copies keeps the L2 cold;
+ * tuning keys for the tcgen05 GEMM: 10 = CTAs a small-M GEMM is split into (0 = one per SM), 11 = maximum
+ * pipeline stages, 12 = allow split-K (1) or not (0). */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1 line 2: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32
@@ -174,10 +180,17 @@ int lsp_scan(lsp_ctx* ctx, const float* score, const int32_t* yhat, const float*
 int lsp_op_linear(lsp_ctx* ctx, int op, const void* A, const void* W, const void* W2, void* out, int M,
                   int N, int K);
 
-/* Device time (ms) of the last step by kernel class, host float[8]:
- * 0 embed+norms, 1 GEMMs, 2 attention, 3 head, 4 merge+scan, 5 commit/append, 6 total, 7 reserved.
- * Only filled when option key 2 (per-class timing, serialises with events) is 1. */
+/* Device time (ms) accumulated since lsp_reset_counters() by kernel class, host float[8]:
+ * 0 embed+norms, 1 layer GEMMs, 2 attention, 3 fused LM head, 4 merge+scan, 5 commit/append, 6 whole steps
+ * (always filled), 7 reserved.  Classes 0-5 are only filled while option key 2 (per-class CUDA-event timing)
+ * is 1.  Synchronises the stream. */
 int lsp_last_timing(lsp_ctx* ctx, float* ms);
+
+/* Host-side accounting since lsp_reset_counters(), host double[8]: 0 kernel launches, 1 layer-GEMM algorithmic
+ * bytes (every operand and result once), 2 layer-GEMM flops, 3 attention bytes (every K/V row once per layer
+ * plus Q and O), 4 KV-append bytes (read + write), 5 LM-head bytes, 6 LM-head flops, 7 denoiser passes. */
+int lsp_get_counters(lsp_ctx* ctx, double* out);
+int lsp_reset_counters(lsp_ctx* ctx);
 
 const char* lsp_last_error(const lsp_ctx* ctx);
 int lsp_destroy(lsp_ctx* ctx);

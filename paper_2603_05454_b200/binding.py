@@ -17,7 +17,7 @@ FLAG_RUN_TO_END, FLAG_NEAR_THRESHOLD, FLAG_NEAR_TIE = 8, 16, 32
 
 EXPORTS = ["lsp_workspace_bytes", "lsp_kv_cache_bytes", "lsp_init", "lsp_set_sched", "lsp_set_option",
            "lsp_begin", "lsp_denoise_step", "lsp_commit", "lsp_generate", "lsp_active", "lsp_score_rows",
-           "lsp_get_scores", "lsp_head_scan", "lsp_scan", "lsp_op_linear", "lsp_last_timing",
+           "lsp_get_scores", "lsp_head_scan", "lsp_scan", "lsp_op_linear", "lsp_last_timing", "lsp_get_counters", "lsp_reset_counters",
            "lsp_last_error", "lsp_destroy"]
 
 
@@ -72,6 +72,8 @@ def _load():
     l.lsp_scan.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int] + [C.c_void_p] * 4
     l.lsp_op_linear.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int]
     l.lsp_last_timing.argtypes = [C.c_void_p, C.c_void_p]
+    l.lsp_get_counters.argtypes = [C.c_void_p, C.c_void_p]
+    l.lsp_reset_counters.argtypes = [C.c_void_p]
     l.lsp_last_error.restype = C.c_char_p
     l.lsp_last_error.argtypes = [C.c_void_p]
     l.lsp_destroy.argtypes = [C.c_void_p]
@@ -254,6 +256,15 @@ class LSPDecoder:
         a = np.zeros(8, dtype=np.float32)
         self._check(lib.lsp_last_timing(self._h, a.ctypes.data))
         return a
+
+    def counters(self):
+        a = np.zeros(8, dtype=np.float64)
+        self._check(lib.lsp_get_counters(self._h, a.ctypes.data))
+        return dict(zip(("launches", "gemm_bytes", "gemm_flops", "attn_bytes", "append_bytes", "head_bytes",
+                         "head_flops", "steps"), a.tolist()))
+
+    def reset_counters(self):
+        self._check(lib.lsp_reset_counters(self._h))
 
     # views of the caller-visible state (device memory owned here)
     def kv_view(self):

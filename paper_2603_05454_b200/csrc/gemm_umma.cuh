@@ -33,7 +33,6 @@ constexpr int UM_MAX_STAGES = 12;
 constexpr uint64_t UM_WAIT_NS = 2000000000ull;   // 2 s
 
 // ---- PTX wrappers -----------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ uint64_t globaltimer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -204,11 +203,88 @@ struct UmmaArgs {
   int num_kb;   // K / 64
   int stages;
   int m_fast;   // 1: blockIdx.x walks the row tiles (keeps one weight tile hot in L2 across the rows), 0: the column tiles
+  int splits;        // split-K factor (blockIdx.z); 1 = none
+  int kb_per_split;  // k-blocks per split (the last split may get fewer)
+  float* scratch;    // split-K partial tiles: [tile][split][128][BN] fp32
+  unsigned* counters;// split-K arrival counters, one per output tile, zero between launches
   unsigned* status;
 };
 
 template <int BN>
 constexpr int umma_stage_bytes() { return UM_BM * UM_BK * 2 + BN * UM_BK * 2; }
+
+// Split-K epilogue: publishes this CTA's partial tile; the CTA that arrives last at the tile sums all partials in
+// split order (deterministic) and runs the fused epilogue.  Returns false when the launch is not split.
+template <int BN, typename Epi>
+__device__ __forceinline__ bool splitk_epilogue(const UmmaArgs& args, const Epi& epi, uint32_t tmem_base, int q, int lane,
+                                                int m, int m0, int tile, volatile uint32_t* epi_last) {
+  if constexpr (Epi::kReduce) {
+    return false;
+  } else {
+    if (args.splits <= 1) return false;
+    constexpr int HALF = BN / 2;
+
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+      const int n_col_tiles = args.m_fast ? gridDim.y : gridDim.x;
+      const int tile_lin = (m0 / UM_BM) * n_col_tiles + tile;
+      const int r_in = q * 32 + lane;
+      float* base = args.scratch + (size_t)tile_lin * args.splits * (UM_BM * BN);
+      float* mine = base + ((size_t)blockIdx.z * UM_BM + r_in) * BN;
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 16) {
+        float v[16];
+        tc_ld16(t_row + c, v);
+        if (m < args.M) {
+          float4* d4 = reinterpret_cast<float4*>(mine + c);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        }
+      }
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (threadIdx.x == 64) {
+        const unsigned old = atomicAdd(args.counters + tile_lin, 1u);
+        if (old == (unsigned)args.splits - 1u) {
+          args.counters[tile_lin] = 0;        // ready for the next launch
+          *epi_last = 1;
+        }
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (*epi_last) {
+        __threadfence();
+        const float* row = base + (size_t)r_in * BN;
+        constexpr int CH = Epi::kDual ? HALF : BN;
+        const int j0 = tile * CH;
+#pragma unroll 1
+        for (int c = 0; c < CH; c += 16) {
+          float a0[16], a1[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
+          if (m < args.M && j0 + c < args.n_pairs) {
+            for (int sp = 0; sp < args.splits; ++sp) {
+              const float4* p0 = reinterpret_cast<const float4*>(row + (size_t)sp * UM_BM * BN + c);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float4 t = __ldcg(p0 + i);
+                a0[4 * i] += t.x; a0[4 * i + 1] += t.y; a0[4 * i + 2] += t.z; a0[4 * i + 3] += t.w;
+              }
+              if (Epi::kDual) {
+                const float4* p1 = reinterpret_cast<const float4*>(row + (size_t)sp * UM_BM * BN + HALF + c);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const float4 t = __ldcg(p1 + i);
+                  a1[4 * i] += t.x; a1[4 * i + 1] += t.y; a1[4 * i + 2] += t.z; a1[4 * i + 3] += t.w;
+                }
+              }
+            }
+            epi16(epi, m, j0 + c, a0, a1);
+          }
+        }
+      }
+    return true;
+  }
+}
 
 template <int BN, typename Epi>
 __global__ void __launch_bounds__(UM_THREADS, 1)
@@ -226,6 +302,8 @@ k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   // bars[0..S) = full, bars[S..2S) = empty, bars[2S] = accumulator ready
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 1);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  volatile uint32_t* epi_fail = tmem_slot + 2;     // set when any epilogue warp's wait expired
+  volatile uint32_t* epi_last = tmem_slot + 3;     // split-K: this CTA arrived last at its tile
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = (args.m_fast ? blockIdx.x : blockIdx.y) * UM_BM;
   const int tile = args.m_fast ? blockIdx.y : blockIdx.x;
@@ -250,6 +328,8 @@ k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     }
     mbar_init(acc_bar, 1);
     *abort_flag = 0;
+    *epi_fail = 0;
+    *epi_last = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -263,7 +343,8 @@ k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int num_kb = args.num_kb;
+  const int kb0 = blockIdx.z * args.kb_per_split;
+  const int num_kb = min(args.kb_per_split, args.num_kb - kb0);
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -280,9 +361,9 @@ k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
         mbar_expect_tx(full_bar(s), STAGE_BYTES);
         const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
-        tma_load_2d(sa, &map_a, kb * UM_BK, m0, full_bar(s));
-        tma_load_2d(sa + A_BYTES, &map_b0, kb * UM_BK, row_b0, full_bar(s));
-        tma_load_2d(sa + A_BYTES + B_HALF_BYTES, &map_b1, kb * UM_BK, row_b1, full_bar(s));
+        tma_load_2d(sa, &map_a, (kb0 + kb) * UM_BK, m0, full_bar(s));
+        tma_load_2d(sa + A_BYTES, &map_b0, (kb0 + kb) * UM_BK, row_b0, full_bar(s));
+        tma_load_2d(sa + A_BYTES + B_HALF_BYTES, &map_b1, (kb0 + kb) * UM_BK, row_b1, full_bar(s));
         ++issued;
       }
       // Do not leave while copies may still be landing in this CTA's shared memory.
@@ -323,9 +404,13 @@ k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     const int q = warp & 3;                        // TMEM lane quarter this warp may access
     const int m = m0 + q * 32 + lane;
     bool ok = mbar_wait(acc_bar, 0u, abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) *epi_fail = 1;
+    asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps agree on the outcome
+    ok = (*epi_fail == 0);
     if (!ok) {
       if (lane == 0 && !*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 3u; }
+    } else if (splitk_epilogue<BN, Epi>(args, epi, tmem_base, q, lane, m, m0, tile, epi_last)) {
+      // handled by the split-K path
     } else {
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -380,6 +465,14 @@ struct UmmaState {
   PFN_encodeTiled encode = nullptr;
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> cache;
   int max_smem = 0;
+  int n_sm = 148;
+  float* scratch = nullptr;        // split-K partial tiles (device), scratch_bytes long
+  size_t scratch_bytes = 0;
+  unsigned* counters = nullptr;    // split-K arrival counters (device), n_counters entries, zero between launches
+  int n_counters = 0;
+  int target_ctas = 0;             // 0 = one CTA per SM
+  int max_stages = UM_MAX_STAGES;
+  int allow_split = 1;
   std::string err;
 };
 
@@ -395,6 +488,7 @@ inline int umma_init(UmmaState& st) {
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&st.max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaDeviceGetAttribute(&st.n_sm, cudaDevAttrMultiProcessorCount, dev);
   return 0;
 }
 
@@ -423,13 +517,15 @@ inline int umma_head_tiles(int vocab) { return (vocab + UM_HEAD_BN - 1) / UM_HEA
 
 template <int BN, typename Epi>
 int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
-                int n_rows_w, const Epi& epi, unsigned* status) {
+                int n_rows_w, const Epi& epi, unsigned* status, int splits) {
   constexpr int stage = umma_stage_bytes<BN>();
   const int aux = 1024 /*alignment slack*/ + 8 * (2 * UM_MAX_STAGES + 1) + 16;
   int stages = (st.max_smem - aux) / stage;
-  if (stages > UM_MAX_STAGES) stages = UM_MAX_STAGES;
+  if (stages > st.max_stages) stages = st.max_stages;
   const int num_kb = K / UM_BK;
-  if (stages > num_kb) stages = num_kb;
+  const int kb_per_split = (num_kb + splits - 1) / splits;
+  splits = (num_kb + kb_per_split - 1) / kb_per_split;      // no empty split
+  if (stages > kb_per_split) stages = kb_per_split;
   if (stages < 1) { st.err = "not enough shared memory"; return -2; }
   const size_t smem = (size_t)stages * stage + aux;
   static bool attr_set = false;   // per instantiation
@@ -447,36 +543,50 @@ int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W
   const int m_fast = Epi::kReduce ? 1 : 0;
   dim3 grid((NP + per_tile - 1) / per_tile, (M + UM_BM - 1) / UM_BM);
   if (m_fast) grid = dim3(grid.y, grid.x);
-  UmmaArgs args{M, NP, K, num_kb, stages, m_fast, status};
+  grid.z = splits;
+  UmmaArgs args{M, NP, K, num_kb, stages, m_fast, splits, kb_per_split, st.scratch, st.counters, status};
   k_gemm_umma<BN, Epi><<<grid, UM_THREADS, smem, stream>>>(*ma, *mb0, *mb1, args, epi);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
   return 0;
 }
 
-// Tile-width choice: the widest tile that still gives every SM a CTA; the rotary epilogue needs both partners of a
-// pair inside one head, which caps the tile at head_dim columns.
+// Tile-width and split-K choice.  Large problems (at least one CTA per SM without splitting) take the widest tile.
+// Small-M problems are bound by streaming the weights once: they take 128-column tiles (so the activation tile is not
+// re-read more often than the weights) and split K until every SM has a CTA.  The rotary epilogue needs both partners
+// of a pair inside one head, which caps the tile at head_dim columns.
 template <typename Epi>
 int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
               int n_rows_w, const Epi& epi, unsigned* status) {
   if (K % UM_BK) { st.err = "K must be a multiple of 64"; return -6; }
   if constexpr (Epi::kReduce) {
-    return umma_launch<UM_HEAD_BN, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+    return umma_launch<UM_HEAD_BN, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 1);
   } else {
     const int cols = Epi::kDual ? 2 * NP : NP;
     const int mt = (M + UM_BM - 1) / UM_BM;
+    const int num_kb = K / UM_BK;
     int max_bn = 256;
     if constexpr (std::is_same<Epi, EpiQKVRope<bf16>>::value) max_bn = 2 * epi.half;
-    int bn = 32;
-    for (int cand = 256; cand >= 32; cand >>= 1) {
-      if (cand > max_bn) continue;
-      if ((long)mt * ((cols + cand - 1) / cand) >= 148) { bn = cand; break; }
+    const int target = st.target_ctas > 0 ? st.target_ctas : st.n_sm;
+    int bn = max_bn, splits = 1;
+    const long big_tiles = (long)mt * ((cols + max_bn - 1) / max_bn);
+    if (big_tiles < target) {
+      bn = Epi::kDual ? max_bn : (max_bn < 128 ? max_bn : 128);
+      const long tiles = (long)mt * ((cols + bn - 1) / bn);
+      if (st.allow_split && st.scratch != nullptr && tiles < target) {
+        splits = (int)((target + tiles / 2) / tiles);
+        if (splits > num_kb / 4) splits = num_kb / 4;
+        if (splits < 1) splits = 1;
+        while (splits > 1 && ((size_t)tiles * splits * UM_BM * bn * sizeof(float) > st.scratch_bytes ||
+                              tiles > st.n_counters))
+          --splits;
+      }
     }
     switch (bn) {
-      case 256: return umma_launch<256, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
-      case 128: return umma_launch<128, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
-      case 64: return umma_launch<64, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
-      default: return umma_launch<32, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+      case 256: return umma_launch<256, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, splits);
+      case 128: return umma_launch<128, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, splits);
+      case 64: return umma_launch<64, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, splits);
+      default: return umma_launch<32, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, splits);
     }
   }
 }

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "../../include/lsp.h"
+#include "attention_mma.cuh"
 #include "attention_simt.cuh"
 #include "gemm_simt.cuh"
 #include "misc_kernels.cuh"
@@ -32,7 +33,7 @@ struct lsp_ctx {
   int max_batch = 0, max_len = 0, max_rows = 0;
   size_t esz = 0;
   cudaStream_t stream = nullptr;
-  int gemm_impl = 1, attn_impl = 1, timing = 0;
+  int gemm_impl = 1, attn_impl = 1, timing = 0, async_ops = 0, op_repeat = 1, op_rotate = 1;
   // workspace carve (device)
   char *X = nullptr, *Nrm = nullptr, *Qb = nullptr, *Att = nullptr, *Hf = nullptr, *stage = nullptr;
   Top2* part = nullptr;
@@ -56,6 +57,10 @@ struct lsp_ctx {
   int last_M = 0;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   float timing_ms[8] = {0};
+  std::vector<cudaEvent_t> seg_ev;      // per-class timing: pairs of events, created on demand
+  std::vector<int> seg_cls;
+  int seg_n = 0;
+  double counters[8] = {0};             // see lsp_get_counters
   std::string err;
 #ifndef LSP_NO_UMMA
   UmmaState umma;
@@ -74,6 +79,39 @@ int fail(lsp_ctx* c, int code, const char* fmt, ...) {
     c->err = buf;
   }
   return code;
+}
+
+enum { CLS_MISC = 0, CLS_GEMM = 1, CLS_ATTN = 2, CLS_HEAD = 3, CLS_SCAN = 4, CLS_COMMIT = 5 };
+enum { CNT_LAUNCHES = 0, CNT_GEMM_BYTES = 1, CNT_GEMM_FLOPS = 2, CNT_ATTN_BYTES = 3, CNT_APPEND_BYTES = 4,
+       CNT_HEAD_BYTES = 5, CNT_HEAD_FLOPS = 6, CNT_STEPS = 7 };
+
+// Opens a timed segment of kernel class cls (only when per-class timing is on).
+void seg_begin(lsp_ctx* c, int cls) {
+  if (!c->timing) return;
+  if ((size_t)(2 * c->seg_n + 2) > c->seg_ev.size()) {
+    cudaEvent_t a, b;
+    cudaEventCreate(&a);
+    cudaEventCreate(&b);
+    c->seg_ev.push_back(a);
+    c->seg_ev.push_back(b);
+    c->seg_cls.push_back(cls);
+  }
+  c->seg_cls[c->seg_n] = cls;
+  cudaEventRecord(c->seg_ev[2 * c->seg_n], c->stream);
+}
+void seg_end(lsp_ctx* c) {
+  if (!c->timing) return;
+  cudaEventRecord(c->seg_ev[2 * c->seg_n + 1], c->stream);
+  c->seg_n += 1;
+}
+// After a stream synchronisation: adds the elapsed time of every closed segment to its class.
+void seg_collect(lsp_ctx* c) {
+  if (!c->timing) return;
+  for (int i = 0; i < c->seg_n; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->seg_ev[2 * i], c->seg_ev[2 * i + 1]) == cudaSuccess) c->timing_ms[c->seg_cls[i]] += ms;
+  }
+  c->seg_n = 0;
 }
 
 #define CU(call)                                                                                   \
@@ -106,8 +144,11 @@ struct Carve {
 
 struct Layout {
   size_t X, Nrm, Qb, Att, Hf, part, yhat, pmax, margin, row_seq, row_pos, head_src, desc, scan, rope, status,
-      stage, total;
+      gemm_scratch, gemm_counters, stage, total;
 };
+
+constexpr size_t kGemmScratchBytes = 64u << 20;   // split-K partial tiles
+constexpr int kGemmCounters = 4096;               // split-K arrival counters
 
 int head_tiles_max(const lsp_model_cfg* m) { return (m->vocab + 63) / 64; }
 
@@ -133,6 +174,8 @@ Layout make_layout(const lsp_model_cfg* m, int max_batch, int max_len) {
   L.scan = cv.take(4 * (size_t)max_batch * 4);
   L.rope = cv.take((size_t)max_len * (m->head_dim / 2) * sizeof(float2));
   L.status = cv.take(256);
+  L.gemm_scratch = cv.take(kGemmScratchBytes);
+  L.gemm_counters = cv.take(kGemmCounters * 4);
   L.stage = cv.take((size_t)m->n_layers * 2 * R * kvd * esz);
   L.total = cv.off;
   return L;
@@ -152,6 +195,17 @@ int check_model(const lsp_model_cfg* m) {
 template <typename T, typename Epi>
 int run_gemm(lsp_ctx* c, const T* A, const T* W0, const T* W1, int M, int NP, int K, int n_rows_w, const Epi& epi) {
   if (M <= 0) return LSP_OK;
+  {
+    // algorithmic work of this launch: every operand and result once
+    const double cols = Epi::kDual ? 2.0 * NP : (double)NP;
+    const double outb = Epi::kReduce ? 16.0 * M : (double)M * NP * sizeof(T);
+    const int k_b = Epi::kReduce ? CNT_HEAD_BYTES : CNT_GEMM_BYTES, k_f = Epi::kReduce ? CNT_HEAD_FLOPS : CNT_GEMM_FLOPS;
+    c->counters[k_b] += (cols * K + (double)M * K) * sizeof(T) + outb;
+    c->counters[k_f] += 2.0 * M * cols * K;
+    c->counters[CNT_LAUNCHES] += 1;
+  }
+  seg_begin(c, Epi::kReduce ? CLS_HEAD : CLS_GEMM);
+  struct SegGuard { lsp_ctx* c; ~SegGuard() { seg_end(c); } } seg_guard{c};
 #ifndef LSP_NO_UMMA
   if constexpr (std::is_same<T, bf16>::value) {
     if (c->gemm_impl == 1) {
@@ -220,6 +274,9 @@ int check_status(lsp_ctx* c) {
   if (c->h_status[0] != 0) {
     const unsigned code = c->h_status[0], where = c->h_status[1];
     cudaMemsetAsync(c->d_status, 0, 16, c->stream);
+#ifndef LSP_NO_UMMA
+    if (c->umma.counters) cudaMemsetAsync(c->umma.counters, 0, (size_t)c->umma.n_counters * 4, c->stream);
+#endif
     cudaStreamSynchronize(c->stream);
     return fail(c, LSP_ERR_DEVICE_TIMEOUT, "device-side bounded wait expired (code %u, site %u)", code, where);
   }
@@ -258,8 +315,11 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   T* Qb = (T*)c->Qb;
   T* Att = (T*)c->Att;
   T* Hf = (T*)c->Hf;
+  seg_begin(c, CLS_MISC);
   k_assemble_embed<T><<<M, 128, 0, c->stream>>>(sd, B, c->tokens, c->tok_stride, m.mask_id, (const T*)c->embed, d, X,
                                                c->row_seq, c->row_pos, c->head_src);
+  seg_end(c);
+  c->counters[CNT_LAUNCHES] += 1;
   CU(cudaGetLastError());
   const size_t plane = (size_t)c->max_rows * kvd;           // elements per staged (layer, K|V) plane
   const size_t cplane = (size_t)c->max_batch * c->max_len * kvd;
@@ -269,7 +329,10 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
     T* stV = stK + plane;
     const T* cK = (const T*)c->kv_cache + (size_t)(2 * l) * cplane;
     const T* cV = cK + cplane;
+    seg_begin(c, CLS_MISC);
     k_rmsnorm<T><<<M, 256, 0, c->stream>>>(X, (const T*)c->attn_norm[l], Nrm, nullptr, d, m.rms_eps);
+    seg_end(c);
+    c->counters[CNT_LAUNCHES] += 1;
     CU(cudaGetLastError());
     {
       EpiQKVRope<T> e{Qb, stK, stV, c->rope_cs, c->row_pos, m.n_heads, m.n_kv_heads, dh / 2};
@@ -278,13 +341,38 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
       if (rc) return rc;
     }
     {
+      // algorithmic attention traffic: every key/value row of every sequence once per layer, plus Q and O
+      for (int b = 0; b < B; ++b) {
+        if (c->N[b] == 0) continue;
+        const double rows_b = c->pend[b] + c->N[b];
+        c->counters[CNT_ATTN_BYTES] += (2.0 * (c->F[b] + rows_b) * kvd + 2.0 * rows_b * qd) * sizeof(T);
+      }
+      c->counters[CNT_LAUNCHES] += 1;
+      seg_begin(c, CLS_ATTN);
+      bool done = false;
+      if constexpr (std::is_same<T, bf16>::value) {
+        if (c->attn_impl == 1) {
+          const int G = m.n_heads / m.n_kv_heads;
+          dim3 g2((maxQ * G + AM_BM - 1) / AM_BM, m.n_kv_heads, B);
+          const float sl2 = scale * 1.4426950408889634f;
+          if (dh == 128)
+            k_attn_mma<128><<<g2, 128, attn_mma_smem_bytes<128>(), c->stream>>>(
+                Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
+          else
+            k_attn_mma<64><<<g2, 128, attn_mma_smem_bytes<64>(), c->stream>>>(
+                Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
+          done = true;
+        }
+      }
       dim3 grid((maxQ + AS_BQ - 1) / AS_BQ, m.n_heads, B);
-      if (dh == 128)
+      if (done) {
+      } else if (dh == 128)
         k_attn_simt<T, 128><<<grid, 128, 0, c->stream>>>(Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
                                                          (size_t)c->max_len * kvd, scale);
       else
         k_attn_simt<T, 64><<<grid, 128, 0, c->stream>>>(Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
                                                         (size_t)c->max_len * kvd, scale);
+      seg_end(c);
       CU(cudaGetLastError());
     }
     {
@@ -292,7 +380,10 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
       const int rc = run_gemm<T>(c, Att, (const T*)c->w_o[l], (const T*)c->w_o[l], M, d, qd, d, e);
       if (rc) return rc;
     }
+    seg_begin(c, CLS_MISC);
     k_rmsnorm<T><<<M, 256, 0, c->stream>>>(X, (const T*)c->ffn_norm[l], Nrm, nullptr, d, m.rms_eps);
+    seg_end(c);
+    c->counters[CNT_LAUNCHES] += 1;
     CU(cudaGetLastError());
     {
       EpiSwiGLU<T> e{Hf, m.d_ffn};
@@ -306,15 +397,23 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
     }
   }
   // masked rows only: final norm (gathered), fused head, merge, scan
+  seg_begin(c, CLS_MISC);
   k_rmsnorm<T><<<Mh, 256, 0, c->stream>>>(X, (const T*)c->final_norm, Nrm, c->head_src, d, m.rms_eps);
+  seg_end(c);
+  c->counters[CNT_LAUNCHES] += 1;
   CU(cudaGetLastError());
   int n_tiles = 0;
   int rc = run_head<T>(c, Nrm, Mh, &n_tiles);
   if (rc) return rc;
+  seg_begin(c, CLS_SCAN);
   rc = run_merge_scan(c, Mh, n_tiles, sd.head_off, B);
+  seg_end(c);
+  c->counters[CNT_LAUNCHES] += 2;
+  c->counters[CNT_STEPS] += 1;
   if (rc) return rc;
   CU(cudaEventRecord(c->ev1, c->stream));
   CU(cudaStreamSynchronize(c->stream));
+  seg_collect(c);
   rc = check_status(c);
   if (rc) return rc;
   float ms = 0.f;
@@ -333,7 +432,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
       rec[b].ms = ms;
     }
   }
-  c->timing_ms[6] = ms;
+  c->timing_ms[6] += ms;
   c->proposed = true;
   c->score_rows = Mh;
   c->last_M = M;
@@ -457,6 +556,7 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
   if (e == cudaSuccess) e = cudaEventCreate(&c->ev0);
   if (e == cudaSuccess) e = cudaEventCreate(&c->ev1);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 256, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws + L.gemm_counters, 0, kGemmCounters * 4, c->stream);
   if (e == cudaSuccess) {
     const int n = max_len * (model->head_dim / 2);
     k_rope_table<<<(n + 255) / 256, 256, 0, c->stream>>>(c->rope_cs, max_len, model->head_dim / 2,
@@ -471,6 +571,12 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
   c->h_status[0] = 0;
 #ifndef LSP_NO_UMMA
   if (model->dtype == 1) {
+    c->umma.scratch = (float*)(ws + L.gemm_scratch);
+    c->umma.scratch_bytes = kGemmScratchBytes;
+    c->umma.counters = (unsigned*)(ws + L.gemm_counters);
+    c->umma.n_counters = kGemmCounters;
+    cudaFuncSetAttribute(k_attn_mma<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_mma_smem_bytes<128>());
+    cudaFuncSetAttribute(k_attn_mma<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_mma_smem_bytes<64>());
     const int urc = umma_init(c->umma);
     if (urc != 0) {
       lsp_destroy(c);
@@ -495,6 +601,14 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   if (key == 0) c->gemm_impl = value;
   else if (key == 1) c->attn_impl = value;
   else if (key == 2) c->timing = value;
+  else if (key == 3) c->async_ops = value;
+  else if (key == 4) c->op_repeat = value < 1 ? 1 : value;
+  else if (key == 5) c->op_rotate = value < 1 ? 1 : value;
+#ifndef LSP_NO_UMMA
+  else if (key == 10) c->umma.target_ctas = value;
+  else if (key == 11) c->umma.max_stages = value < 1 ? 1 : (value > UM_MAX_STAGES ? UM_MAX_STAGES : value);
+  else if (key == 12) c->umma.allow_split = value;
+#endif
   else return fail(c, LSP_ERR_ARG, "lsp_set_option: unknown key %d", key);
   return LSP_OK;
 }
@@ -561,9 +675,14 @@ int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
   if (chunks < 1) chunks = 1;
   if (chunks > 64) chunks = 64;
   dim3 grid(chunks, m.n_layers * 2, B);
+  seg_begin(c, CLS_COMMIT);
   k_commit_append<<<grid, 256, 0, c->stream>>>(desc_of(c), (const uint4*)c->stage, (uint4*)c->kv_cache,
                                                stage_plane_v4, cache_plane_v4, cache_seq_v4, row_v4, c->yhat,
                                                c->tokens, c->tok_stride);
+  seg_end(c);
+  c->counters[CNT_LAUNCHES] += 1;
+  for (int b = 0; b < B; ++b)
+    if (c->N[b] > 0) c->counters[CNT_APPEND_BYTES] += 2.0 * c->pend[b] * kvd * c->esz * 2.0 * m.n_layers;
   CU(cudaGetLastError());
   for (int b = 0; b < B; ++b) {
     if (c->N[b] == 0) continue;
@@ -633,7 +752,11 @@ int lsp_head_scan(lsp_ctx* c, const void* hidden, const int32_t* seq_offsets, in
   rc = c->m.dtype == 0 ? run_head<float>(c, (const float*)hidden, rows, &n_tiles)
                        : run_head<bf16>(c, (const bf16*)hidden, rows, &n_tiles);
   if (rc) return rc;
+  seg_begin(c, CLS_SCAN);
   rc = run_merge_scan(c, rows, n_tiles, c->d_desc + 4 * (c->max_batch + 1), batch);
+  seg_end(c);
+  c->counters[CNT_LAUNCHES] += 2;
+  c->counters[CNT_STEPS] += 1;
   if (rc) return rc;
   c->score_rows = rows;
   return scan_outputs(c, batch, l_run, l_commit, flags, tau_used);
@@ -660,9 +783,16 @@ int lsp_op_linear(lsp_ctx* c, int op, const void* A, const void* W, const void* 
   if (!c || !A || !W || !out || M < 0 || N < 1 || K < 1) return LSP_ERR_ARG;
   if (op < 0 || op > 2 || (op == 2 && !W2)) return fail(c, LSP_ERR_ARG, "lsp_op_linear: bad op");
   if (K % 64 || N % 16) return fail(c, LSP_ERR_SHAPE, "lsp_op_linear: K must be a multiple of 64 and N of 16");
-  const int rc = c->m.dtype == 0 ? op_linear_impl<float>(c, op, A, W, W2, out, M, N, K)
-                                 : op_linear_impl<bf16>(c, op, A, W, W2, out, M, N, K);
+  int rc = 0;
+  for (int r = 0; r < c->op_repeat && rc == 0; ++r) {
+    const size_t off = (size_t)(r % c->op_rotate) * N * K * c->esz;
+    const void* w = (const char*)W + off;
+    const void* w2 = W2 ? (const char*)W2 + off : nullptr;
+    rc = c->m.dtype == 0 ? op_linear_impl<float>(c, op, A, w, w2, out, M, N, K)
+                         : op_linear_impl<bf16>(c, op, A, w, w2, out, M, N, K);
+  }
   if (rc) return rc;
+  if (c->async_ops) return LSP_OK;
   CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
   CU(cudaStreamSynchronize(c->stream));
   return check_status(c);
@@ -670,7 +800,24 @@ int lsp_op_linear(lsp_ctx* c, int op, const void* A, const void* W, const void* 
 
 int lsp_last_timing(lsp_ctx* c, float* ms) {
   if (!c || !ms) return LSP_ERR_ARG;
+  CU(cudaStreamSynchronize(c->stream));
+  seg_collect(c);
   memcpy(ms, c->timing_ms, sizeof c->timing_ms);
+  return LSP_OK;
+}
+
+int lsp_get_counters(lsp_ctx* c, double* out) {
+  if (!c || !out) return LSP_ERR_ARG;
+  memcpy(out, c->counters, sizeof c->counters);
+  return LSP_OK;
+}
+
+int lsp_reset_counters(lsp_ctx* c) {
+  if (!c) return LSP_ERR_ARG;
+  cudaStreamSynchronize(c->stream);
+  seg_collect(c);
+  memset(c->counters, 0, sizeof c->counters);
+  memset(c->timing_ms, 0, sizeof c->timing_ms);
   return LSP_OK;
 }
 
@@ -683,6 +830,7 @@ int lsp_destroy(lsp_ctx* c) {
   if (c->h_status) cudaFreeHost(c->h_status);
   if (c->ev0) cudaEventDestroy(c->ev0);
   if (c->ev1) cudaEventDestroy(c->ev1);
+  for (cudaEvent_t e : c->seg_ev) cudaEventDestroy(e);
   delete c;
   return LSP_OK;
 }
