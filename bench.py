@@ -1,0 +1,477 @@
+#!/usr/bin/env python
+"""Benchmark of the LSP decode hot path on B200:  python bench.py --gpus N --steps K --warmup W
+
+One *step* is one whole LSP decode (Algorithm 1: every denoiser pass, fused LM-head confidence reduction, scan,
+commit and KV append) of one batch of the workload.  The default workload is the LLaDA-8B-shaped full decode
+("cfg3": 32 layers, d 4096, 32x128 heads, FFN 12288, vocab 126464, bf16, batch 1, prompt 256 + 256 masked,
+tau 0.9, delimiters 1..32); `--workload cfg4|cfg5|cfg2` selects the Dream-7B-shaped decode, the long batched
+decode or the head-only configuration.  Weights and prompts are seeded synthetic values (random init).
+
+Prints ONE JSON line:
+  value          committed tokens/s over the K timed decodes, inputs resident in HBM (CUDA events, max over ranks)
+  e2e            the same through lsp_generate_host: prompt copied from pinned host memory and the finished token
+                 buffer copied back inside the timed region, every decode
+  roofline       the dominant kernel class of the workload (layer GEMMs), algorithmic bytes / kernel time, measured
+                 with per-launch CUDA events in a second pass over the same K decodes
+  classes        the same figures for every kernel class (attention, LM head, append, ...)
+  cpu_baseline   the CPU oracle timed on a bounded sample of the same workload (rank 0, N = 1 only)
+  also           a shorter run of the Dream-7B-shaped decode (cfg4), whose passes are tensor-bound
+
+`--impl reference` times the CPU oracle alone (there is no other reference implementation of this path).
+With N > 1 (torchrun) every rank runs an independent replica of the workload with its own prompts: the path has
+no exchange step, so there is no collective on it; only the timing is reduced (max) across ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+CLASSES = ("misc", "gemm", "attn", "head", "scan", "commit")
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures summarised under
+# profiles/, keyed by kernel class, with the hash of the kernel sources they were taken on.  A class whose sources
+# changed since reports null.
+NCU_TRAFFIC = {}
+
+
+def source_hash():
+    h = hashlib.sha1()
+    d = os.path.join(ROOT, "paper_2603_05454_b200", "csrc")
+    for f in sorted(os.listdir(d)):
+        h.update(open(os.path.join(d, f), "rb").read())
+    return h.hexdigest()[:12]
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return json.load(open(p)), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid = uuid
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", self.uuid, "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.strip() == "Active":
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm_sorted = sorted(sm)
+        return {"sm_mhz": sm_sorted[len(sm_sorted) // 2], "sm_max_mhz": max(mx), "power_w_max": max(pw),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 0) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------------------------------------------------
+# CPU oracle legs (the only place this file executes oracle/)
+# ------------------------------------------------------------------------------------------------------------
+ORACLE_LAYERS = 1     # depth of the model slice the oracle sample runs
+ORACLE_STEPS = 2      # denoiser steps of the decode the sample covers
+
+
+def oracle_sample_setup(wl, gen_device):
+    """Builds the oracle model for a slice (first ORACLE_LAYERS layers, full widths and vocabulary) of the workload's
+    model and the prompt of sequence 0.  Input values come from the shared seeded generator."""
+    import dataclasses
+    import lsp_synth as S
+    from oracle import dlm
+    sh = dataclasses.replace(wl.shape, n_layers=min(ORACLE_LAYERS, wl.shape.n_layers))
+    w = S.make_weights(sh, 0, device=gen_device)
+    om = dlm.OracleDLM(sh, w)
+    del w
+    prompt = S.make_prompt(1, wl.prompt_len, sh, 0)[0].numpy()
+    return sh, om, prompt
+
+
+def oracle_sample_run(wl, om, prompt):
+    """ORACLE_STEPS steps of the oracle's decode of one sequence.  Returns (seconds, tokens committed)."""
+    import numpy as np
+    from oracle.decode import decode, make_is_delim
+    t0 = time.perf_counter()
+    _, recs, _ = decode(om, prompt, wl.gen_len, make_is_delim(*wl.delim),
+                        dict(tau=float(np.float32(wl.tau))), max_steps=ORACLE_STEPS)
+    dt = time.perf_counter() - t0
+    return dt, sum(r["L_commit"] for r in recs)
+
+
+def oracle_sample_text(wl):
+    return (f"oracle.decode, first {ORACLE_STEPS} denoiser steps of one sequence of {wl.name} "
+            f"(prompt {wl.prompt_len} + {wl.gen_len} masked) on a {ORACLE_LAYERS}-layer slice of the model "
+            f"(full widths and vocabulary); value = tokens it committed / (seconds x n_layers/{ORACLE_LAYERS}), "
+            "i.e. scaled to the full depth (the head's share is scaled too, so a lower bound on the oracle's rate)")
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle as it stands, on the host cores."""
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import lsp_synth as S
+    wl = S.config(args.workload if args.workload != "cfg2" else "cfg3")
+    gen_device = "cuda:0" if torch.cuda.is_available() else "cpu"
+    sh, om, prompt = oracle_sample_setup(wl, gen_device)
+    scale = wl.shape.n_layers / sh.n_layers
+    for _ in range(args.warmup):
+        oracle_sample_run(wl, om, prompt)
+    t, tok = 0.0, 0
+    for _ in range(args.steps):
+        dt, n = oracle_sample_run(wl, om, prompt)
+        t += dt
+        tok += n
+    value = tok / (t * scale)
+    cores = blas_threads()
+    line = {"impl": "reference", "metric": "committed_tokens_per_s", "value": value, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "batch": 1, "prompt_len": wl.prompt_len, "gen_len": wl.gen_len,
+                       "tau": wl.tau, "step": "one bounded oracle sample"},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": oracle_sample_text(wl)},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------------------
+# the CUDA path
+# ------------------------------------------------------------------------------------------------------------
+def class_report(cnt, tms, peaks):
+    """Per-class achieved bandwidth / throughput from the library's work counters and per-launch event times."""
+    hbm = peaks["hbm_gbs"]
+    tc = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    src = source_hash()
+    out = {}
+    work = {"gemm": (cnt["gemm_bytes"], cnt["gemm_flops"]), "attn": (cnt["attn_bytes"], cnt["attn_flops"]),
+            "head": (cnt["head_bytes"], cnt["head_flops"]), "commit": (cnt["append_bytes"], 0.0)}
+    for i, name in enumerate(CLASSES):
+        ms = float(tms[i])
+        n = cnt["launches_" + name]
+        e = {"launches": int(n), "ms_total": round(ms, 3), "us_per_launch": round(1e3 * ms / n, 3) if n else None}
+        if name in work and ms > 0:
+            b, f = work[name]
+            e["gbs"] = round(b / (ms * 1e-3) / 1e9, 1)
+            e["hbm_frac"] = round(e["gbs"] / hbm, 4)
+            if f:
+                e["tflops"] = round(f / (ms * 1e-3) / 1e12, 1)
+                e["tensor_frac_sustained"] = round(e["tflops"] / tc, 4)
+            e["bytes_per_launch"] = round(b / n) if n else None
+        t = NCU_TRAFFIC.get(name)
+        e["traffic"] = t["bytes_per_launch"] if t and t.get("src") == src else None
+        out[name] = e
+    return out
+
+
+def run_decode_bench(wl, dev, rank, world, peaks, steps, warmup, sampler=None, with_e2e=True):
+    import numpy as np
+    import torch
+    import lsp_synth as S
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+
+    sh = wl.shape
+    B, P, G = wl.batch, wl.prompt_len, wl.gen_len
+    w = S.make_weights(sh, 0, device=dev)
+    bm = S.delimiter_bitmap(sh.vocab, *wl.delim).to(dev)
+    dec = LSPDecoder(sh, w, SchedCfg(tau=wl.tau, delim_bitmap=bm), B, P + G, device=dev)
+    prompt = S.make_prompt(B, P, sh, 100 + rank)           # every replica decodes its own prompts
+    host_in = torch.zeros(B, P + G, dtype=torch.int32).pin_memory()
+    host_in[:, :P] = prompt
+    host_out = torch.zeros(B, P + G, dtype=torch.int32).pin_memory()
+    tokens = torch.zeros(B, P + G, dtype=torch.int32, device=dev)
+    tokens.copy_(host_in)
+    Pl, Gl = [P] * B, [G] * B
+
+    def decode_resident():
+        dec.begin(tokens, Pl, Gl)
+        n, _ = dec.generate()
+        return n
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(warmup):
+        decode_resident()
+    assert int((tokens == sh.mask_id).sum()) == 0, "decode left masked positions"
+    dec.reset_counters()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    if sampler:
+        sampler.start()
+    ev0.record()
+    passes = 0
+    for _ in range(steps):
+        passes += decode_resident()
+    ev1.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms = ev0.elapsed_time(ev1)
+    cnt = dec.counters()
+    res = {"ms": ms, "passes": passes, "launches": int(cnt["launches"]), "clocks": clocks, "tokens": B * G * steps}
+
+    if with_e2e:
+        for _ in range(min(warmup, 2)):
+            dec.generate_host(tokens, host_in, host_out, Pl, Gl)
+        barrier()
+        ev0.record()
+        for _ in range(steps):
+            dec.generate_host(tokens, host_in, host_out, Pl, Gl)
+        ev1.record()
+        barrier()
+        res["e2e_ms"] = ev0.elapsed_time(ev1)
+        res["h2d"] = host_in.numel() * 4
+        res["d2h"] = host_out.numel() * 4
+        assert int((host_out == sh.mask_id).sum()) == 0 and bool((host_out[:, :P] == host_in[:, :P]).all())
+
+    # second pass over the same decodes with one CUDA-event pair around every launch (per-class kernel time)
+    dec.set_option(2, 1)
+    decode_resident()
+    dec.reset_counters()
+    for _ in range(steps):
+        decode_resident()
+    tms = dec.last_timing()
+    cnt2 = dec.counters()
+    dec.set_option(2, 0)
+    res["classes"] = class_report(cnt2, tms, peaks)
+    # per-step profile of one more decode (rows shrink as the prefix grows)
+    dec.begin(tokens, Pl, Gl)
+    n, recs = dec.generate(max_recs=B * (G + 1))
+    rows_ms = {}
+    for i in range(0, len(recs), B):
+        rows = sum(r["rows"] for r in recs[i:i + B])
+        rows_ms.setdefault(rows, []).append(recs[i]["ms"])
+    ks = sorted(rows_ms)
+    pick = [ks[0], ks[len(ks) // 2], ks[-1]] if ks else []
+    res["step_ms_by_rows"] = {str(k): round(float(np.median(rows_ms[k])), 4) for k in pick}
+    live = [r["L_commit"] for r in recs if r["n_before"] > 0]
+    res["l_commit_mean"] = float(np.mean(live)) if live else None
+    dec.close()
+    del dec, w
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_head_bench(dev, peaks, steps, warmup):
+    """cfg2: the fused LM head + confidence reduction + scan alone on [8 x 1024, 4096] hidden states."""
+    import numpy as np
+    import torch
+    import lsp_synth as S
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+    d, V, B, L = 4096, 126464, 8, 1024
+    sh = S.ModelShape(1, d, 32, 32, 128, 64, V, dtype="bf16", head_scale=6.0)
+    z = lambda *s: torch.zeros(*s, dtype=torch.bfloat16, device=dev)
+    w = dict(embed=z(8, d), w_head=S.normal((V, d), 0, S.TID_HEAD, 0.02 * 6.0, torch.bfloat16, dev),
+             final_norm=torch.ones(d, dtype=torch.bfloat16, device=dev),
+             layers=[dict(attn_norm=z(d), w_qkv=z(3 * d, d), w_o=z(d, d), ffn_norm=z(d), w_gate=z(64, d), w_up=z(64, d),
+                          w_down=z(d, 64))])
+    bm = S.delimiter_bitmap(V, 1, 32).to(dev)
+    dec = LSPDecoder(sh, w, SchedCfg(tau=0.9, delim_bitmap=bm), B, L, device=dev)
+    hidden = S.normal((B * L, d), 0, 77, 1.0, torch.bfloat16, dev)
+    host_h = hidden.cpu().pin_memory()
+    off = np.arange(B + 1, dtype=np.int32) * L
+    for _ in range(warmup):
+        dec.head_scan(hidden, off)
+    dec.reset_counters()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize(dev)
+    ev0.record()
+    for _ in range(steps):
+        dec.head_scan(hidden, off)
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    ms = ev0.elapsed_time(ev1)
+    cnt = dec.counters()
+    ev0.record()
+    for _ in range(steps):
+        hidden.copy_(host_h, non_blocking=True)
+        dec.head_scan(hidden, off)
+        dec.scores()
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    e2e_ms = ev0.elapsed_time(ev1)
+    dec.set_option(2, 1)
+    dec.head_scan(hidden, off)
+    dec.reset_counters()
+    for _ in range(steps):
+        dec.head_scan(hidden, off)
+    tms = dec.last_timing()
+    cnt2 = dec.counters()
+    dec.close()
+    return dict(ms=ms, e2e_ms=e2e_ms, launches=int(cnt["launches"]), positions=B * L * steps,
+                h2d=host_h.numel() * 2, d2h=B * L * 12, classes=class_report(cnt2, tms, peaks))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="own", choices=["own", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--also", default="cfg4", help="second workload reported under 'also' at N=1 ('none' to skip)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import lsp_synth as S
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=dev)
+    peaks, peak_kind = load_peaks()
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    sampler = ClockSampler(uuid)
+
+    if args.workload == "cfg2":
+        sampler.start()
+        r = run_head_bench(dev, peaks, args.steps, args.warmup)
+        clocks = sampler.stop()
+        head = r["classes"]["head"]
+        line = {"metric": "scored_positions_per_s", "value": r["positions"] / (r["ms"] * 1e-3), "unit": "positions/s",
+                "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms"] / args.steps,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "cfg2: fused LM head + confidence + LSP scan, hidden [8,1024,4096], vocab 126464",
+                           "l2": "inputs_exceed_l2 (1.04 GB head weight)"},
+                "roofline": {"bound": "tensor", "achieved": head.get("tflops"), "peak": peaks["bf16_tflops"],
+                             "unit": "TFLOP/s", "frac": (head.get("tflops") or 0) / peaks["bf16_tflops"],
+                             "traffic": head.get("traffic"), "peak_kind": "burst, of " + peak_kind},
+                "e2e": {"value": r["positions"] / (r["e2e_ms"] * 1e-3), "unit": "positions/s",
+                        "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"]},
+                "gpu_launches": r["launches"], "classes": r["classes"], "clocks": clocks}
+        print(json.dumps(line))
+        return 0
+
+    wl = S.config(args.workload)
+    r = run_decode_bench(wl, dev, rank, world, peaks, args.steps, args.warmup, sampler)
+    ms = torch.tensor([r["ms"], r.get("e2e_ms", 0.0)], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(ms, op=torch.distributed.ReduceOp.MAX)
+    ms_max, e2e_max = float(ms[0]), float(ms[1])
+    tokens_total = r["tokens"] * world
+    value = tokens_total / (ms_max * 1e-3)
+    gemm = r["classes"]["gemm"]
+    line = {"metric": "committed_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_max / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{wl.name}: LSP decode, {wl.shape.n_layers} layers d={wl.shape.d_model} "
+                                   f"heads {wl.shape.n_heads}/{wl.shape.n_kv_heads}x{wl.shape.head_dim} ffn "
+                                   f"{wl.shape.d_ffn} vocab {wl.shape.vocab}, random init",
+                       "batch": wl.batch, "prompt_len": wl.prompt_len, "gen_len": wl.gen_len, "tau": wl.tau,
+                       "delimiters": list(wl.delim), "head_scale": wl.shape.head_scale, "snap_window": 16,
+                       "step": "one full decode (all denoiser passes)", "parallelism": f"replicas x{world}",
+                       "l2": "inputs_exceed_l2 (every pass streams the full weight set, far larger than the 126 MB L2)"},
+            "denoiser_passes_per_decode": r["passes"] / args.steps,
+            "ms_per_denoiser_step": ms_max / r["passes"],
+            "ms_per_denoiser_step_by_rows": r["step_ms_by_rows"],
+            "tokens_per_pass": r["l_commit_mean"],
+            "roofline": {"bound": "hbm", "achieved": gemm.get("gbs"), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gemm.get("hbm_frac"), "traffic": gemm.get("traffic"),
+                         "kernel": "k_gemm_umma (layer projections and FFN; weight-streaming regime, rows <= 512)",
+                         "peak_kind": "of " + peak_kind,
+                         "timed": "per-launch CUDA events, second pass over the same K decodes"},
+            "classes": r["classes"],
+            "e2e": {"value": tokens_total / (e2e_max * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": r["h2d"],
+                    "d2h_bytes_per_step": r["d2h"]},
+            "gpu_launches": r["launches"], "clocks": r["clocks"]}
+
+    if rank == 0 and world == 1 and args.also != "none" and args.also != args.workload:
+        wl2 = S.config(args.also)
+        k2 = max(1, min(2, args.steps))
+        r2 = run_decode_bench(wl2, dev, 0, 1, peaks, k2, 3, None, with_e2e=False)
+        g2 = r2["classes"]["gemm"]
+        line["also"] = [{"workload": wl2.name, "batch": wl2.batch, "prompt_len": wl2.prompt_len, "gen_len": wl2.gen_len,
+                         "head_scale": wl2.shape.head_scale, "tau": wl2.tau, "steps": k2,
+                         "value": r2["tokens"] / (r2["ms"] * 1e-3), "unit": "tokens/s",
+                         "denoiser_passes_per_decode": r2["passes"] / k2,
+                         "ms_per_denoiser_step": r2["ms"] / r2["passes"],
+                         "ms_per_denoiser_step_by_rows": r2["step_ms_by_rows"],
+                         "roofline": {"bound": "tensor", "achieved": g2.get("tflops"),
+                                      "peak": peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                                      "unit": "TFLOP/s", "frac": g2.get("tensor_frac_sustained"),
+                                      "traffic": g2.get("traffic"), "peak_kind": "sustained, of " + peak_kind},
+                         "classes": r2["classes"]}]
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sh, om, prompt = oracle_sample_setup(wl, dev)
+        dt, tok = oracle_sample_run(wl, om, prompt)
+        scale = wl.shape.n_layers / sh.n_layers
+        line["cpu_baseline"] = {"value": tok / (dt * scale), "unit": "tokens/s", "cores": blas_threads(),
+                                "kind": "oracle", "sample": oracle_sample_text(wl), "seconds": round(dt, 3)}
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -3,10 +3,10 @@
  *
  * The library runs the per-step hot path of the LSP scheduler for diffusion language models:
  * one bidirectional denoiser pass over [pending block | masked suffix] with the committed prefix
- * served from a contiguous KV cache (Algorithm 1 line 4), the fused LM-head + confidence
- * reduction (Eq. 1 and the softmax max-probability; line 5), the longest-stable-run scan with
- * adaptive threshold (Eq. 2), delimiter snap and fallback (lines 6-8), and the atomic commit with
- * the contiguous KV append (lines 9-10).
+ * served from a contiguous KV cache (Algorithm 1, the forward pass), the fused LM-head + confidence
+ * reduction (Eq. 1 and the softmax max-probability), the longest-stable-run scan with
+ * adaptive threshold (Eq. 2), delimiter snap and fallback (Sec. 3.2), and the atomic commit with
+ * the contiguous KV append (Algorithm 1, commit and AppendToCache).
  *
  * Conventions
  *  - Every function returns 0 on success or a negative LSP_ERR_* code; lsp_last_error() gives text.
@@ -129,27 +129,37 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * pipeline stages, 12 = allow split-K (1) or not (0). */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
-/* Algorithm 1 line 2: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32
+/* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32
  * [batch, token_stride], caller-owned, prompt ids already at [0, prompt_len[b]); the library writes
  * mask_id over [prompt_len[b], prompt_len[b]+gen_len[b]) and later the committed ids.  prompt_len,
  * gen_len: host [batch].  prompt_len[b] >= 1, gen_len[b] >= 1, sum <= max_len, <= token_stride. */
 int lsp_begin(lsp_ctx* ctx, int32_t* tokens, int token_stride, const int32_t* prompt_len,
               const int32_t* gen_len, int batch);
 
-/* Algorithm 1 lines 4-8 for every unfinished sequence: the pass, the scores, the scan; proposes L
+/* Algorithm 1, forward pass through fallback, for every unfinished sequence: the pass, the scores, the scan; proposes L
  * and changes no committed state.  rec: host [batch] or NULL.  Synchronises the stream. */
 int lsp_denoise_step(lsp_ctx* ctx, lsp_step_rec* rec);
 
-/* Algorithm 1 lines 9-10: writes yhat_{1:L} into the token buffer, appends the pending block's K/V
+/* Algorithm 1, commit and AppendToCache: writes yhat_{1:L} into the token buffer, appends the pending block's K/V
  * (computed by the last pass) to the cache as one contiguous copy per layer, and makes the new
  * block pending.  L_override: host [batch] (entries of finished sequences ignored) or NULL to use the
  * proposed lengths.  Needs a preceding lsp_denoise_step; 1 <= L <= N_b else LSP_ERR_STATE and nothing
  * changes.  Asynchronous. */
 int lsp_commit(lsp_ctx* ctx, const int32_t* L_override);
 
-/* Algorithm 1 lines 3-11: step + commit until every sequence is fully committed.  recs: host
+/* Algorithm 1, the whole loop: step + commit until every sequence is fully committed.  recs: host
  * [max_recs] records in (step, sequence) order, or NULL; n_steps: number of denoiser passes. */
 int lsp_generate(lsp_ctx* ctx, lsp_step_rec* recs, int max_recs, int* n_steps);
+
+/* Algorithm 1 from host memory: copies tokens_in (host int32 [batch, token_stride], prompt ids at
+ * [0, prompt_len[b]) of every row; pinned or pageable) into the caller's device buffer tokens (device int32
+ * [batch, token_stride], scratch the caller owns), runs lsp_begin + lsp_generate, and copies the finished
+ * buffer (prompt followed by the committed ids) to tokens_out (host, same shape; may equal tokens_in).
+ * Both copies run on the context's stream; the call returns after the result has arrived.  Errors as
+ * lsp_begin / lsp_generate; on error tokens_out is not written. */
+int lsp_generate_host(lsp_ctx* ctx, int32_t* tokens, int token_stride, const int32_t* tokens_in,
+                      int32_t* tokens_out, const int32_t* prompt_len, const int32_t* gen_len, int batch,
+                      lsp_step_rec* recs, int max_recs, int* n_steps);
 
 /* Number of still-active positions per sequence (host [batch]); returns the count of unfinished sequences
  * through *n_unfinished. */
@@ -186,9 +196,11 @@ int lsp_op_linear(lsp_ctx* ctx, int op, const void* A, const void* W, const void
  * is 1.  Synchronises the stream. */
 int lsp_last_timing(lsp_ctx* ctx, float* ms);
 
-/* Host-side accounting since lsp_reset_counters(), host double[8]: 0 kernel launches, 1 layer-GEMM algorithmic
+/* Host-side accounting since lsp_reset_counters(), host double[16]: 0 kernel launches, 1 layer-GEMM algorithmic
  * bytes (every operand and result once), 2 layer-GEMM flops, 3 attention bytes (every K/V row once per layer
- * plus Q and O), 4 KV-append bytes (read + write), 5 LM-head bytes, 6 LM-head flops, 7 denoiser passes. */
+ * plus Q and O), 4 KV-append bytes (read + write), 5 LM-head bytes, 6 LM-head flops, 7 denoiser passes,
+ * 8..13 kernel launches by class (same classes as lsp_last_timing 0..5), 14 attention flops
+ * (4 * queries * keys * n_heads * head_dim per layer), 15 committed tokens. */
 int lsp_get_counters(lsp_ctx* ctx, double* out);
 int lsp_reset_counters(lsp_ctx* ctx);
 

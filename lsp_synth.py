@@ -220,12 +220,12 @@ def config(name: str) -> Workload:
         return Workload(name, ModelShape(2, 256, 4, 4, 64, 1024, 2048, dtype="fp32", head_scale=8.0),
                         1, 32, 64, 0.9, (1, 8))
     if name == "cfg3":
-        return Workload(name, ModelShape(32, 4096, 32, 32, 128, 12288, 126464, head_scale=3.0),
+        return Workload(name, ModelShape(32, 4096, 32, 32, 128, 12288, 126464, head_scale=12.0),
                         1, 256, 256, 0.9, (1, 32))
     if name == "cfg4":
         return Workload(name, ModelShape(28, 3584, 28, 4, 128, 18944, 152064, rope_theta=1e6,
-                                         head_scale=3.0), 4, 512, 512, 0.85, (1, 64))
+                                         head_scale=12.0), 4, 512, 512, 0.85, (1, 64))
     if name == "cfg5":
-        return Workload(name, ModelShape(32, 4096, 32, 32, 128, 12288, 126464, head_scale=3.0),
+        return Workload(name, ModelShape(32, 4096, 32, 32, 128, 12288, 126464, head_scale=12.0),
                         16, 1024, 1024, 0.9, (1, 32))
     raise KeyError(name)

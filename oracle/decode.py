@@ -41,7 +41,7 @@ def decode(model, prompt, gen_len, is_delim, policy, score="pmax", use_cache=Tru
     F, Fp, pend, N = 0, P, P, G        # cache rows, token boundary, pending block, active length
     recs = []
     step = 0
-    while N > 0:                                                        # Alg. 1 line 3
+    while N > 0:                                                        # Alg. 1: loop      
         if use_cache:
             ids = np.concatenate([tokens[F:F + pend], np.full(N, s.mask_id)])
             pos = np.arange(F, F + pend + N)
@@ -52,21 +52,21 @@ def decode(model, prompt, gen_len, is_delim, policy, score="pmax", use_cache=Tru
             pos = np.arange(0, Fp + N)
             head_rows = np.arange(Fp, Fp + N)
             ck, cv = model.empty_cache()
-        logits, k_new, v_new = model.forward(ids, pos, ck, cv, head_rows)   # line 4
-        yhat, pmax, delta = scores_from_logits(logits, s.mask_id if exclude_mask else -1)  # line 5
+        logits, k_new, v_new = model.forward(ids, pos, ck, cv, head_rows)   # pass  
+        yhat, pmax, delta = scores_from_logits(logits, s.mask_id if exclude_mask else -1)  # scores
         sc = pmax if score == "pmax" else delta
-        r = _scan.lsp_scan(sc, yhat, is_delim, margin=delta, **policy)      # lines 6-8
+        r = _scan.lsp_scan(sc, yhat, is_delim, margin=delta, **policy)      # tau, snap
         L = r["L_commit"]
         rec = dict(step=step, n_before=N, rows=len(ids), F=F, Fp=Fp, pend=pend, yhat=yhat,
                    pmax=pmax, delta=delta, **r)
         if on_step is not None:
             on_step(rec, logits, k_new, v_new)
-        if use_cache:                                                   # line 10 (lagged)
+        if use_cache:                                                   # append (lagged) 
             for l in range(s.n_layers):
                 cache_k[l] = np.concatenate([cache_k[l], k_new[l][:pend]], axis=0)
                 cache_v[l] = np.concatenate([cache_v[l], v_new[l][:pend]], axis=0)
             F += pend
-        tokens[Fp:Fp + L] = yhat[:L]                                    # line 9
+        tokens[Fp:Fp + L] = yhat[:L]                                    # commit
         Fp += L
         pend = L
         N -= L

@@ -1,4 +1,4 @@
-"""Oracle: one denoiser pass p_theta(X_F, X_A; K) (Algorithm 1 line 4) for the transformer
+"""Oracle: one denoiser pass p_theta(X_F, X_A; K) (Algorithm 1, the forward pass) for the transformer
 shape the benchmark configurations fix (the paper treats the model as a black box): a
 pre-norm bidirectional transformer with RMSNorm, rotary positions (rotate-half pairing),
 multi-head / grouped-query attention without any mask, SwiGLU feed-forward, no biases and an

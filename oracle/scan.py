@@ -1,12 +1,12 @@
 """Oracle: stability run, adaptive threshold, delimiter snap, fallback (Sec. 3.2, Eq. 2, the
-snapping display formula, Algorithm 1 lines 5-8).  TEST INFRASTRUCTURE, not a product path.
+snapping display formula, Algorithm 1, threshold / snap / fallback steps).  TEST INFRASTRUCTURE, not a product path.
 
 Notation follows the paper: positions of the active suffix are 1..N, ``score_i`` is the
 stability score (logit margin delta_i of Eq. 1, or the max-probability used by the benchmark
 configurations), ``L'`` the candidate run, ``L`` the committed length, ``D`` the delimiter
 set, ``W`` the look-back window, ``L_min`` the minimum block.
 
-Readings taken where the paper is silent or inconsistent (all also listed in the design notes):
+Readings taken where the paper is silent or inconsistent:
   * the test is ``score_i >= tau`` (the paper says "exceed"; ">=" is what makes tau = 0
     accept everything for either score);
   * adaptive mode picks the LARGEST achievable m in [ceil(alpha N), floor(beta N)]; when no m

@@ -1,5 +1,5 @@
 """Oracle: per-position prediction and stability scores from a row of logits (Sec. 3.2, Eq. 1;
-Algorithm 1 line 5).  TEST INFRASTRUCTURE, not a product path.
+Algorithm 1, the score step).  TEST INFRASTRUCTURE, not a product path.
 
   yhat  = argmax_v z_v            (ties -> lowest id; the paper is silent)
   delta = z_(1) - z_(2)           (Eq. 1: difference of the two largest LOGITS; z_(2) is the

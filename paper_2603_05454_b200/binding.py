@@ -16,7 +16,7 @@ FLAG_SNAPPED, FLAG_FALLBACK, FLAG_RANGE_UNACHIEVABLE = 1, 2, 4
 FLAG_RUN_TO_END, FLAG_NEAR_THRESHOLD, FLAG_NEAR_TIE = 8, 16, 32
 
 EXPORTS = ["lsp_workspace_bytes", "lsp_kv_cache_bytes", "lsp_init", "lsp_set_sched", "lsp_set_option",
-           "lsp_begin", "lsp_denoise_step", "lsp_commit", "lsp_generate", "lsp_active", "lsp_score_rows",
+           "lsp_begin", "lsp_denoise_step", "lsp_commit", "lsp_generate", "lsp_generate_host", "lsp_active", "lsp_score_rows",
            "lsp_get_scores", "lsp_head_scan", "lsp_scan", "lsp_op_linear", "lsp_last_timing", "lsp_get_counters", "lsp_reset_counters",
            "lsp_last_error", "lsp_destroy"]
 
@@ -65,6 +65,8 @@ def _load():
     l.lsp_denoise_step.argtypes = [C.c_void_p, C.POINTER(StepRec)]
     l.lsp_commit.argtypes = [C.c_void_p, C.c_void_p]
     l.lsp_generate.argtypes = [C.c_void_p, C.POINTER(StepRec), C.c_int, C.POINTER(C.c_int)]
+    l.lsp_generate_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                    C.POINTER(StepRec), C.c_int, C.POINTER(C.c_int)]
     l.lsp_active.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]
     l.lsp_score_rows.argtypes = [C.c_void_p]
     l.lsp_get_scores.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -210,6 +212,25 @@ class LSPDecoder:
         out = [_rec(r) for r in recs][: n.value * self.batch] if recs is not None else []
         return n.value, out
 
+    def generate_host(self, tokens_dev: torch.Tensor, tokens_in: torch.Tensor, tokens_out: torch.Tensor, prompt_len,
+                      gen_len, max_recs: int = 0):
+        """Algorithm 1 from host memory: tokens_in / tokens_out are CPU int32 tensors [batch, stride] (pinned or
+        not), tokens_dev the device buffer of the same shape the decode runs in."""
+        assert tokens_dev.dtype == torch.int32 and tokens_dev.is_cuda and tokens_dev.is_contiguous()
+        for t in (tokens_in, tokens_out):
+            assert t.dtype == torch.int32 and not t.is_cuda and t.is_contiguous() and t.shape == tokens_dev.shape
+        self.tokens = tokens_dev
+        self.batch = tokens_dev.shape[0]
+        pl = np.ascontiguousarray(prompt_len, dtype=np.int32)
+        gl = np.ascontiguousarray(gen_len, dtype=np.int32)
+        n = C.c_int(0)
+        recs = (StepRec * max_recs)() if max_recs else None
+        self._check(lib.lsp_generate_host(self._h, tokens_dev.data_ptr(), tokens_dev.shape[1], tokens_in.data_ptr(),
+                                          tokens_out.data_ptr(), pl.ctypes.data, gl.ctypes.data, self.batch, recs,
+                                          max_recs, C.byref(n)))
+        out = [_rec(r) for r in recs][: n.value * self.batch] if recs is not None else []
+        return n.value, out
+
     def active(self):
         a = np.zeros(self.batch, dtype=np.int32)
         u = C.c_int(0)
@@ -258,10 +279,11 @@ class LSPDecoder:
         return a
 
     def counters(self):
-        a = np.zeros(8, dtype=np.float64)
+        a = np.zeros(16, dtype=np.float64)
         self._check(lib.lsp_get_counters(self._h, a.ctypes.data))
         return dict(zip(("launches", "gemm_bytes", "gemm_flops", "attn_bytes", "append_bytes", "head_bytes",
-                         "head_flops", "steps"), a.tolist()))
+                         "head_flops", "steps", "launches_misc", "launches_gemm", "launches_attn", "launches_head",
+                         "launches_scan", "launches_commit", "attn_flops", "tokens"), a.tolist()))
 
     def reset_counters(self):
         self._check(lib.lsp_reset_counters(self._h))

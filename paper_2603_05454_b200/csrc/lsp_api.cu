@@ -60,7 +60,7 @@ struct lsp_ctx {
   std::vector<cudaEvent_t> seg_ev;      // per-class timing: pairs of events, created on demand
   std::vector<int> seg_cls;
   int seg_n = 0;
-  double counters[8] = {0};             // see lsp_get_counters
+  double counters[16] = {0};            // see lsp_get_counters
   std::string err;
 #ifndef LSP_NO_UMMA
   UmmaState umma;
@@ -83,7 +83,14 @@ int fail(lsp_ctx* c, int code, const char* fmt, ...) {
 
 enum { CLS_MISC = 0, CLS_GEMM = 1, CLS_ATTN = 2, CLS_HEAD = 3, CLS_SCAN = 4, CLS_COMMIT = 5 };
 enum { CNT_LAUNCHES = 0, CNT_GEMM_BYTES = 1, CNT_GEMM_FLOPS = 2, CNT_ATTN_BYTES = 3, CNT_APPEND_BYTES = 4,
-       CNT_HEAD_BYTES = 5, CNT_HEAD_FLOPS = 6, CNT_STEPS = 7 };
+       CNT_HEAD_BYTES = 5, CNT_HEAD_FLOPS = 6, CNT_STEPS = 7, CNT_CLS_LAUNCHES = 8 /* + class, 6 entries */,
+       CNT_ATTN_FLOPS = 14, CNT_TOKENS = 15 };
+
+// Counts n kernel launches of class cls.
+void count_launch(lsp_ctx* c, int cls, int n = 1) {
+  c->counters[CNT_LAUNCHES] += n;
+  c->counters[CNT_CLS_LAUNCHES + cls] += n;
+}
 
 // Opens a timed segment of kernel class cls (only when per-class timing is on).
 void seg_begin(lsp_ctx* c, int cls) {
@@ -202,7 +209,7 @@ int run_gemm(lsp_ctx* c, const T* A, const T* W0, const T* W1, int M, int NP, in
     const int k_b = Epi::kReduce ? CNT_HEAD_BYTES : CNT_GEMM_BYTES, k_f = Epi::kReduce ? CNT_HEAD_FLOPS : CNT_GEMM_FLOPS;
     c->counters[k_b] += (cols * K + (double)M * K) * sizeof(T) + outb;
     c->counters[k_f] += 2.0 * M * cols * K;
-    c->counters[CNT_LAUNCHES] += 1;
+    count_launch(c, Epi::kReduce ? CLS_HEAD : CLS_GEMM);
   }
   seg_begin(c, Epi::kReduce ? CLS_HEAD : CLS_GEMM);
   struct SegGuard { lsp_ctx* c; ~SegGuard() { seg_end(c); } } seg_guard{c};
@@ -319,7 +326,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   k_assemble_embed<T><<<M, 128, 0, c->stream>>>(sd, B, c->tokens, c->tok_stride, m.mask_id, (const T*)c->embed, d, X,
                                                c->row_seq, c->row_pos, c->head_src);
   seg_end(c);
-  c->counters[CNT_LAUNCHES] += 1;
+  count_launch(c, CLS_MISC);
   CU(cudaGetLastError());
   const size_t plane = (size_t)c->max_rows * kvd;           // elements per staged (layer, K|V) plane
   const size_t cplane = (size_t)c->max_batch * c->max_len * kvd;
@@ -332,7 +339,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
     seg_begin(c, CLS_MISC);
     k_rmsnorm<T><<<M, 256, 0, c->stream>>>(X, (const T*)c->attn_norm[l], Nrm, nullptr, d, m.rms_eps);
     seg_end(c);
-    c->counters[CNT_LAUNCHES] += 1;
+    count_launch(c, CLS_MISC);
     CU(cudaGetLastError());
     {
       EpiQKVRope<T> e{Qb, stK, stV, c->rope_cs, c->row_pos, m.n_heads, m.n_kv_heads, dh / 2};
@@ -346,8 +353,9 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
         if (c->N[b] == 0) continue;
         const double rows_b = c->pend[b] + c->N[b];
         c->counters[CNT_ATTN_BYTES] += (2.0 * (c->F[b] + rows_b) * kvd + 2.0 * rows_b * qd) * sizeof(T);
+        c->counters[CNT_ATTN_FLOPS] += 4.0 * rows_b * (c->F[b] + rows_b) * qd;
       }
-      c->counters[CNT_LAUNCHES] += 1;
+      count_launch(c, CLS_ATTN);
       seg_begin(c, CLS_ATTN);
       bool done = false;
       if constexpr (std::is_same<T, bf16>::value) {
@@ -383,7 +391,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
     seg_begin(c, CLS_MISC);
     k_rmsnorm<T><<<M, 256, 0, c->stream>>>(X, (const T*)c->ffn_norm[l], Nrm, nullptr, d, m.rms_eps);
     seg_end(c);
-    c->counters[CNT_LAUNCHES] += 1;
+    count_launch(c, CLS_MISC);
     CU(cudaGetLastError());
     {
       EpiSwiGLU<T> e{Hf, m.d_ffn};
@@ -400,7 +408,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   seg_begin(c, CLS_MISC);
   k_rmsnorm<T><<<Mh, 256, 0, c->stream>>>(X, (const T*)c->final_norm, Nrm, c->head_src, d, m.rms_eps);
   seg_end(c);
-  c->counters[CNT_LAUNCHES] += 1;
+  count_launch(c, CLS_MISC);
   CU(cudaGetLastError());
   int n_tiles = 0;
   int rc = run_head<T>(c, Nrm, Mh, &n_tiles);
@@ -408,7 +416,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   seg_begin(c, CLS_SCAN);
   rc = run_merge_scan(c, Mh, n_tiles, sd.head_off, B);
   seg_end(c);
-  c->counters[CNT_LAUNCHES] += 2;
+  count_launch(c, CLS_SCAN, 2);
   c->counters[CNT_STEPS] += 1;
   if (rc) return rc;
   CU(cudaEventRecord(c->ev1, c->stream));
@@ -680,13 +688,14 @@ int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
                                                stage_plane_v4, cache_plane_v4, cache_seq_v4, row_v4, c->yhat,
                                                c->tokens, c->tok_stride);
   seg_end(c);
-  c->counters[CNT_LAUNCHES] += 1;
+  count_launch(c, CLS_COMMIT);
   for (int b = 0; b < B; ++b)
     if (c->N[b] > 0) c->counters[CNT_APPEND_BYTES] += 2.0 * c->pend[b] * kvd * c->esz * 2.0 * m.n_layers;
   CU(cudaGetLastError());
   for (int b = 0; b < B; ++b) {
     if (c->N[b] == 0) continue;
     c->F[b] += c->pend[b];
+    c->counters[CNT_TOKENS] += L[b];
     c->Fp[b] += L[b];
     c->pend[b] = L[b];
     c->N[b] -= L[b];
@@ -714,6 +723,23 @@ int lsp_generate(lsp_ctx* c, lsp_step_rec* recs, int max_recs, int* n_steps) {
   }
   CU(cudaStreamSynchronize(c->stream));
   if (n_steps) *n_steps = steps;
+  return LSP_OK;
+}
+
+int lsp_generate_host(lsp_ctx* c, int32_t* tokens, int token_stride, const int32_t* tokens_in, int32_t* tokens_out,
+                      const int32_t* prompt_len, const int32_t* gen_len, int batch, lsp_step_rec* recs, int max_recs,
+                      int* n_steps) {
+  if (!c || !tokens || !tokens_in || !tokens_out || !prompt_len || !gen_len) return LSP_ERR_ARG;
+  if (batch < 1 || batch > c->max_batch || token_stride < 2)
+    return fail(c, LSP_ERR_ARG, "lsp_generate_host: batch %d not in [1, %d] or bad stride", batch, c->max_batch);
+  const size_t bytes = (size_t)batch * token_stride * sizeof(int32_t);
+  CU(cudaMemcpyAsync(tokens, tokens_in, bytes, cudaMemcpyHostToDevice, c->stream));
+  int rc = lsp_begin(c, tokens, token_stride, prompt_len, gen_len, batch);
+  if (rc) return rc;
+  rc = lsp_generate(c, recs, max_recs, n_steps);
+  if (rc) return rc;
+  CU(cudaMemcpyAsync(tokens_out, tokens, bytes, cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaStreamSynchronize(c->stream));
   return LSP_OK;
 }
 
@@ -755,7 +781,7 @@ int lsp_head_scan(lsp_ctx* c, const void* hidden, const int32_t* seq_offsets, in
   seg_begin(c, CLS_SCAN);
   rc = run_merge_scan(c, rows, n_tiles, c->d_desc + 4 * (c->max_batch + 1), batch);
   seg_end(c);
-  c->counters[CNT_LAUNCHES] += 2;
+  count_launch(c, CLS_SCAN, 2);
   c->counters[CNT_STEPS] += 1;
   if (rc) return rc;
   c->score_rows = rows;

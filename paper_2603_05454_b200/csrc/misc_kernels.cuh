@@ -5,7 +5,7 @@
 namespace lsp {
 
 // ---------------------------------------------------------------------------------------------
-// Row assembly + embedding (Algorithm 1 line 4's input): packed row r of sequence b is position
+// Row assembly + embedding (input of Algorithm 1's forward pass): packed row r of sequence b is position
 // F_b + j; the first pend_b rows carry the tokens committed by the previous step, the rest [MASK].
 // One block per row.  Also fills row_seq / row_pos and the list of rows that go through the LM head.
 // ---------------------------------------------------------------------------------------------
@@ -85,7 +85,7 @@ __global__ void k_merge_partials(const Top2* __restrict__ part, int n_tiles, int
 //   adaptive mode : prefix minimum pm; m is achievable iff pm[m] > pm[m+1]; the largest achievable
 //                   m in [ceil(alpha N), floor(beta N)] is taken, tau = pm[m] (Eq. 2)
 //   snap          : last delimiter j <= L' with L' - j <= W, else the run's end; L' = N commits all;
-//                   L = min(N, max(L, L_min, 1))                               (Algorithm 1 lines 7-8)
+//                   L = min(N, max(L, L_min, 1))                               (Algorithm 1: snap, fallback)
 // ---------------------------------------------------------------------------------------------
 struct ScanParams {
   int mode;
@@ -195,7 +195,7 @@ __global__ void k_lsp_scan(const float* __restrict__ score, const int32_t* __res
 }
 
 // ---------------------------------------------------------------------------------------------
-// Commit (Algorithm 1 lines 9-10).  grid = (chunks, n_layers * 2, batch):
+// Commit (Algorithm 1: commit and AppendToCache).  grid = (chunks, n_layers * 2, batch):
 //   * the pending block's K/V rows, staged by the last pass at packed rows [row_off_b, row_off_b + pend_b),
 //     are copied to cache rows [F_b, F_b + pend_b): one contiguous 128-bit-vector copy per (layer, K|V, b);
 //   * block (0, 0, b) also writes yhat_{1:L_b} into the token buffer at [Fp_b, Fp_b + L_b).
