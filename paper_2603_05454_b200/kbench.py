@@ -85,21 +85,48 @@ def bench_head(M, V, d, reps=10, head_scale=6.0):
                 gbs=round(c["head_bytes"] / reps / us / 1e3, 1), tflops=round(c["head_flops"] / reps / us / 1e6, 1))
 
 
-def bench_decode(name, decodes=1):
+def _fast_weights(sh):
+    """Same shapes and scales as lsp_synth.make_weights, filled by torch's generator in a few launches (profiling
+    aid: a run under a profiler pays for every launch, the seeded generator takes thousands)."""
+    g = torch.Generator(device=DEV)
+    g.manual_seed(0)
+    rnd = lambda *s, std=sh.w_std: torch.empty(*s, dtype=torch.bfloat16, device=DEV).normal_(0.0, std, generator=g)
+    d, hq, hkv, dh, f, v = sh.d_model, sh.n_heads, sh.n_kv_heads, sh.head_dim, sh.d_ffn, sh.vocab
+    one = lambda: torch.ones(d, dtype=torch.bfloat16, device=DEV)
+    return dict(embed=rnd(v, d), w_head=rnd(v, d, std=sh.w_std * sh.head_scale), final_norm=one(),
+                layers=[dict(w_qkv=rnd((hq + 2 * hkv) * dh, d), w_o=rnd(d, hq * dh), w_gate=rnd(f, d), w_up=rnd(f, d),
+                             w_down=rnd(d, f), attn_norm=one(), ffn_norm=one()) for _ in range(sh.n_layers)])
+
+
+def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False):
+    """Per-class kernel times of a decode.  layers > 0 cuts the model to its first layers, max_passes > 0 stops each
+    decode after that many denoiser passes (both are profiling aids: fewer launches, same kernels and row counts)."""
     wl = S.config(name)
     sh = wl.shape
+    if layers > 0:
+        sh.n_layers = layers
     B, P, G = wl.batch, wl.prompt_len, wl.gen_len
-    w = S.make_weights(sh, 0, device=DEV)
+    w = _fast_weights(sh) if fast_init else S.make_weights(sh, 0, device=DEV)
     dec = LSPDecoder(sh, w, SchedCfg(tau=wl.tau, delim_bitmap=S.delimiter_bitmap(sh.vocab, *wl.delim).to(DEV)), B, P + G,
                      device=DEV)
     tokens = torch.zeros(B, P + G, dtype=torch.int32, device=DEV)
     tokens[:, :P] = S.make_prompt(B, P, sh, 100).to(DEV)
-    dec.begin(tokens, [P] * B, [G] * B)
-    dec.generate()
+
+    def run():
+        dec.begin(tokens, [P] * B, [G] * B)
+        if max_passes <= 0:
+            return dec.generate()[0]
+        n = 0
+        while n < max_passes and dec.active()[1] > 0:
+            dec.denoise_step()
+            dec.commit()
+            n += 1
+        return n
+
+    run()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    dec.begin(tokens, [P] * B, [G] * B)
-    n_plain = dec.generate()[0]
+    n_plain = run()
     e1.record()
     torch.cuda.synchronize()
     plain_ms = e0.elapsed_time(e1)
@@ -107,8 +134,7 @@ def bench_decode(name, decodes=1):
     dec.reset_counters()
     n = 0
     for _ in range(decodes):
-        dec.begin(tokens, [P] * B, [G] * B)
-        n += dec.generate()[0]
+        n += run()
     t = dec.last_timing()
     c = dec.counters()
     dec.close()
@@ -135,6 +161,9 @@ def main():
     ap.add_argument("--reps", type=int, default=50)
     ap.add_argument("--copies", type=int, default=0)
     ap.add_argument("--workload", default="cfg3")
+    ap.add_argument("--layers", type=int, default=0)
+    ap.add_argument("--max-passes", type=int, default=0)
+    ap.add_argument("--fast-init", action="store_true")
     ap.add_argument("--opt", type=int, nargs=2, action="append", default=[], help="lsp_set_option key value")
     a = ap.parse_args()
     if a.what == "gemm":
@@ -144,7 +173,7 @@ def main():
         for m in a.M:
             print(json.dumps(bench_head(m, a.V, a.d, a.reps)), flush=True)
     else:
-        print(json.dumps(bench_decode(a.workload)), flush=True)
+        print(json.dumps(bench_decode(a.workload, 1, a.layers, a.max_passes, a.fast_init)), flush=True)
 
 
 if __name__ == "__main__":
