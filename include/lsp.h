@@ -126,7 +126,11 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * key 4 = lsp_op_linear enqueues the operation this many times (timing aid); key 5 = repetition r reads its weights
  * at W + (r mod value) * N * K elements, so a buffer of several weight copies keeps the L2 cold;
  * tuning keys for the tcgen05 GEMM: 10 = CTAs a small-M GEMM is split into (0 = one per SM), 11 = maximum
- * pipeline stages, 12 = allow split-K (1) or not (0). */
+ * pipeline stages, 12 = allow split-K (1) or not (0), 13 = CTAs per SM a weight-streaming GEMM (M <= 128) aims for,
+ * 14 = fewest pipeline stages it accepts for that, 15 = its tile width for plain epilogues (32, 64 or 128),
+ * 16 = GEMMs with at most 128 rows use the persistent weight-streaming kernel (1, default) or the tiled one (0),
+ * 17 = grid of that kernel (0 by row count, 1 one CTA per SM with even shares, 2 a multiple of the tile count),
+ * 18 = row count up to which mode 0 takes even shares. */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

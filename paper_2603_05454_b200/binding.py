@@ -10,7 +10,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "liblsp_b200.so")
+_LIB_PATH = os.environ.get("LSP_LIB") or os.path.join(_HERE, "liblsp_b200.so")   # LSP_LIB: another build of the library
 
 FLAG_SNAPPED, FLAG_FALLBACK, FLAG_RANGE_UNACHIEVABLE = 1, 2, 4
 FLAG_RUN_TO_END, FLAG_NEAR_THRESHOLD, FLAG_NEAR_TIE = 8, 16, 32

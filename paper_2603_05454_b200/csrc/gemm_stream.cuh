@@ -1,0 +1,413 @@
+// Weight-streaming bf16 GEMM for at most 128 activation rows (the shrinking suffix of late decode steps), tcgen05.
+//
+//   acc[m, c] = sum_k A[m, k] * Wt[c, k]        same operands, tiles and fused epilogues as gemm_umma.cuh
+//
+// With M <= 128 a layer GEMM is bound by reading its weights from HBM once, so the kernel is built around one
+// uninterrupted stream of weight tiles per SM:
+//   * persistent CTAs, at most one per SM; the (column tile, K chunk) units of the whole problem are dealt out in
+//     equal contiguous shares (a share may start and end in the middle of a tile), in a single wave;
+//   * a pipeline stage holds 128 elements of K (two 128-byte swizzle atoms per operand): 256 contiguous bytes per
+//     weight row and stage, which on B200 streams at 5.3 TB/s where 128 bytes per row and stage reach only 3.7 TB/s;
+//   * only the activation rows that exist are loaded (a box of 8..128 rows); the MMA still spans 128 accumulator rows,
+//     and the rows past the box, computed from whatever the stage holds, are never stored;
+//   * accumulators are double-buffered in tensor memory, so the epilogue of one tile overlaps the loads and MMAs of
+//     the next; only the first fill and the last epilogue of a CTA are exposed;
+//   * a tile that spans several CTAs is finished by the CTA that arrives last at the tile's counter: every
+//     contributor writes its fp32 partial tile to scratch, and the finisher sums all of them in CTA order (the same
+//     order whoever finishes, so results are deterministic) before running the fused epilogue.
+// Warp roles as in gemm_umma.cuh: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = epilogue.
+// Every wait is bounded; on expiry the kernel records (code, site) in the status word, drains and returns.
+#pragma once
+#include "gemm_umma.cuh"
+
+namespace lsp {
+
+constexpr int ST_BK = 128;                 // K elements per stage (two swizzle atoms)
+constexpr int ST_MAX_STAGES = 8;
+
+struct StreamArgs {
+  int M;            // activation rows (<= 128)
+  int n_pairs;      // dual: pair indices; plain: output columns
+  int n_tiles;      // column tiles
+  int kc;           // K / 128 chunks per tile
+  int a_rows;       // activation box rows (8..128, power of two)
+  int stages;
+  float* scratch;   // [gridDim.x][2][128][BN] fp32 partial tiles
+  unsigned* counters;  // one per column tile, zero between launches
+  unsigned* status;
+};
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// first unit of CTA g when U units are dealt to G CTAs
+__device__ __forceinline__ long st_first_unit(long U, int G, int g) { return U * g / G; }
+// CTA that owns unit u
+__device__ __forceinline__ int st_owner(long U, int G, long u) { return (int)(((u + 1) * G + U - 1) / U) - 1; }
+
+template <int BN, typename Epi>
+__global__ void __launch_bounds__(UM_THREADS, 1)
+k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
+              const __grid_constant__ CUtensorMap map_b1, StreamArgs args, Epi epi) {
+  extern __shared__ uint8_t smem_raw[];
+  constexpr int HALF = BN / 2;
+  constexpr int B_HALF_ATOM = HALF * 128;               // bytes of one half-tile atom (64 K elements)
+  constexpr int B_ATOM = BN * 128;
+  const int A_ATOM = args.a_rows * 128;
+  const int STAGE_BYTES = 2 * (A_ATOM + B_ATOM);
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int S = args.stages;
+  // the barriers sit behind the stages and 16 KB of padding the MMA may read (never written) past the last stage
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * STAGE_BYTES + 16384);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  volatile uint32_t* epi_flag = tmem_slot + 2;          // epilogue warps: this CTA finishes the tile
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar_base = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+  auto accf_bar = [&](int b) { return bar_base + 8u * (2 * S + b); };
+  auto acce_bar = [&](int b) { return bar_base + 8u * (2 * S + 2 + b); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(accf_bar(b), 1);
+      mbar_init(acce_bar(b), 4);
+    }
+    *abort_flag = 0;
+    *epi_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"((uint32_t)(2 * BN))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int G = gridDim.x, g = blockIdx.x;
+  const long U = (long)args.n_tiles * args.kc;
+  const long u0 = st_first_unit(U, G, g), u1 = st_first_unit(U, G, g + 1);
+
+  if (warp == 0) {
+    // ---------------- TMA producer: one uninterrupted stream over this CTA's units ----------------
+    if (lane == 0) {
+      long issued = 0;
+      for (long u = u0; u < u1; ++u) {
+        const int it = (int)(u - u0), s = it % S;
+        const uint32_t ph = (uint32_t)(it / S) & 1u;
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
+          if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 11u; }
+          break;
+        }
+        const int tile = (int)(u / args.kc), c = (int)(u % args.kc);
+        int row_b0, row_b1;
+        if (Epi::kDual) { row_b0 = epi.row0(tile * HALF); row_b1 = epi.row1(tile * HALF); }
+        else { row_b0 = tile * BN; row_b1 = tile * BN + HALF; }
+        mbar_expect_tx(full_bar(s), STAGE_BYTES);
+        const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
+        const uint32_t sb = sa + 2 * A_ATOM;
+        const int k0 = c * ST_BK;
+        // weights first, both atoms of a row group back to back: 256 contiguous bytes per weight row
+        tma_load_2d(sb, &map_b0, k0, row_b0, full_bar(s));
+        tma_load_2d(sb + B_ATOM, &map_b0, k0 + 64, row_b0, full_bar(s));
+        tma_load_2d(sb + B_HALF_ATOM, &map_b1, k0, row_b1, full_bar(s));
+        tma_load_2d(sb + B_ATOM + B_HALF_ATOM, &map_b1, k0 + 64, row_b1, full_bar(s));
+        tma_load_2d(sa, &map_a, k0, 0, full_bar(s));
+        tma_load_2d(sa + A_ATOM, &map_a, k0 + 64, 0, full_bar(s));
+        ++issued;
+      }
+      // do not leave while copies may still be landing in this CTA's shared memory
+      const long first = issued > S ? issued - S : 0;
+      for (long it = first; it < issued; ++it) {
+        volatile uint32_t no_abort = 0;
+        mbar_wait(full_bar((int)(it % S)), (uint32_t)(it / S) & 1u, &no_abort);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(BN);
+      int seg = 0;
+      bool ok = true;
+      for (long u = u0; u < u1 && ok;) {
+        const int tile = (int)(u / args.kc);
+        const long seg_end = min(u1, (long)(tile + 1) * args.kc);
+        const int buf = seg & 1;
+        // wait until the epilogue has drained this accumulator buffer (its previous use was segment seg - 2)
+        if (seg >= 2 && !mbar_wait(acce_bar(buf), (uint32_t)((seg >> 1) - 1) & 1u, abort_flag)) {
+          if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 12u; }
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        bool first = true;
+        for (; u < seg_end; ++u) {
+          const int it = (int)(u - u0), s = it % S;
+          const uint32_t ph = (uint32_t)(it / S) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag)) {
+            if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 13u; }
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
+          const uint32_t sb = sa + 2 * A_ATOM;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const uint64_t da = make_smem_desc(sa + j * A_ATOM);
+            const uint64_t db = make_smem_desc(sb + j * B_ATOM);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              tc_mma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, first ? 0u : 1u);
+              first = false;
+            }
+          }
+          tc_commit(empty_bar(s));
+        }
+        if (ok) tc_commit(accf_bar(buf));
+        ++seg;
+      }
+    }
+  } else {
+    // ---------------- epilogue (warps 2..5) ----------------
+    const int q = warp & 3;
+    const int r_in = q * 32 + lane;
+    const int m = r_in;
+    int seg = 0;
+    bool ok = true;
+    for (long u = u0; u < u1 && ok; ++seg) {
+      const int tile = (int)(u / args.kc);
+      const long tile_u0 = (long)tile * args.kc;
+      const long seg_end = min(u1, tile_u0 + args.kc);
+      const bool whole = (u == tile_u0) && (seg_end == tile_u0 + args.kc);
+      const int buf = seg & 1;
+      if (!mbar_wait(accf_bar(buf), (uint32_t)(seg >> 1) & 1u, abort_flag)) {
+        if (lane == 0 && !*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 14u; }
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
+      bool finish = whole;
+      int g_lo = g, g_hi = g;
+      if (!whole) {
+        // publish this CTA's partial tile, then count its chunks in; the CTA that completes the count finishes the tile
+        // partial tile layout: [16-column chunk][quarter][row][4 floats], so that the lanes of a warp (consecutive
+        // rows) write and read consecutive 16-byte pieces
+        float4* mine = reinterpret_cast<float4*>(args.scratch + (size_t)(g * 2 + (seg == 0 ? 0 : 1)) * UM_BM * BN) + r_in;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 16) {
+          float v[16];
+          tc_ld16(t_row + c, v);
+          if (m < args.M) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              mine[(size_t)((c >> 4) * 4 + i) * UM_BM] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          }
+        }
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (threadIdx.x == 64) {
+          const unsigned add = (unsigned)(seg_end - u);
+          const unsigned old = atomicAdd(args.counters + tile, add);
+          const bool last = (old + add == (unsigned)args.kc);
+          if (last) args.counters[tile] = 0;          // ready for the next launch
+          *epi_flag = last ? 1u : 0u;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        finish = (*epi_flag != 0);
+        if (finish) {
+          __threadfence();
+          g_lo = st_owner(U, G, tile_u0);
+          g_hi = st_owner(U, G, tile_u0 + args.kc - 1);
+        }
+      }
+      // the accumulator buffer is free once every warp has read it (whole tiles read it below)
+      if (!whole) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(buf));
+      }
+      constexpr int CH = Epi::kDual ? HALF : BN;   // pair indices (dual) or columns (plain) per tile
+      const int j0 = tile * CH;
+      if (finish && whole) {
+        // the accumulator is complete in tensor memory: each thread owns one row
+        Top2 red = top2_empty();
+#pragma unroll 1
+        for (int c = 0; c < CH; c += 16) {
+          float a0[16], a1[16];
+          tc_ld16(t_row + c, a0);
+          if (Epi::kDual) tc_ld16(t_row + HALF + c, a1);
+          if constexpr (Epi::kReduce) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int col = j0 + c + i;
+              if (epi.valid(col)) top2_push(red, a0[i], col);
+            }
+          } else {
+            if (m < args.M && j0 + c < args.n_pairs) epi16(epi, m, j0 + c, a0, a1);
+          }
+        }
+        if constexpr (Epi::kReduce) {
+          if (m < args.M) epi.part[(size_t)m * epi.n_tiles + tile] = red;
+        }
+      } else if (finish) {
+        // the tile is the sum of the contributors' partial tiles in scratch.  Work items are (row, 16-column chunk),
+        // dealt over the 128 epilogue threads so that a tile with few rows still uses all of them, and every item
+        // issues the loads of up to four contributors before it adds them (in CTA order: deterministic).
+        constexpr int NCH = CH / 16;                 // chunks per row
+        constexpr int RPP = 128 / NCH;               // rows per pass
+        const int et = threadIdx.x - 64;
+        // plain epilogues: consecutive lanes take consecutive rows (coalesced reads of the partials); the reducing
+        // epilogue keeps a row's chunks in neighbouring lanes so that they can be merged with shuffles
+        const int ch = Epi::kReduce ? et % NCH : et / RPP, c = ch * 16;
+        for (int mm0 = 0; mm0 < args.M; mm0 += RPP) {
+          const int mm = mm0 + (Epi::kReduce ? et / NCH : et % RPP);
+          const bool valid = mm < args.M;
+          float a0[16], a1[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
+          if (valid) {
+            for (int gb = g_lo; gb <= g_hi; gb += 4) {
+              float4 t0[4][4], t1[4][4];
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                const int gg = gb + x;
+                if (gg <= g_hi) {
+                  // contributor gg's segment of this tile is its first one iff its share starts inside the tile
+                  const int slot = (st_first_unit(U, G, gg) >= tile_u0) ? 0 : 1;
+                  const float4* base = reinterpret_cast<const float4*>(args.scratch + (size_t)(gg * 2 + slot) * UM_BM * BN) + mm;
+                  const float4* p0 = base + (size_t)(c >> 4) * 4 * UM_BM;
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) t0[x][i] = __ldcg(p0 + (size_t)i * UM_BM);
+                  if (Epi::kDual) {
+                    const float4* p1 = base + (size_t)((HALF + c) >> 4) * 4 * UM_BM;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) t1[x][i] = __ldcg(p1 + (size_t)i * UM_BM);
+                  }
+                }
+              }
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                if (gb + x <= g_hi) {
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    a0[4 * i] += t0[x][i].x; a0[4 * i + 1] += t0[x][i].y; a0[4 * i + 2] += t0[x][i].z; a0[4 * i + 3] += t0[x][i].w;
+                    if (Epi::kDual) {
+                      a1[4 * i] += t1[x][i].x; a1[4 * i + 1] += t1[x][i].y; a1[4 * i + 2] += t1[x][i].z; a1[4 * i + 3] += t1[x][i].w;
+                    }
+                  }
+                }
+              }
+            }
+          }
+          if constexpr (Epi::kReduce) {
+            Top2 red = top2_empty();
+            if (valid) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const int col = j0 + c + i;
+                if (epi.valid(col)) top2_push(red, a0[i], col);
+              }
+            }
+#pragma unroll
+            for (int o = 1; o < NCH; o <<= 1) red = top2_merge(red, top2_shfl_xor(red, o));
+            if (valid && ch == 0) epi.part[(size_t)mm * epi.n_tiles + tile] = red;
+          } else {
+            if (valid && j0 + c < args.n_pairs) epi16(epi, mm, j0 + c, a0, a1);
+          }
+        }
+      }
+      if (whole) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(buf));
+      }
+      u = seg_end;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * BN)) : "memory");
+  }
+}
+
+// ---- host side ------------------------------------------------------------------------------------------------
+// Scratch the streaming kernel needs for a grid of n_ctas CTAs and tile width bn.
+inline size_t stream_scratch_bytes(int n_ctas, int bn) { return (size_t)n_ctas * 2 * UM_BM * bn * sizeof(float); }
+
+// Number of CTAs.  Dealing the units evenly over all SMs balances the weight stream perfectly but splits almost every
+// tile between two CTAs, which costs a partial tile written and read back per split (M x BN x 4 bytes each way).
+// With at most as many tiles as SMs, a grid that is a multiple of the tile count splits each tile into equal K slices
+// instead (no split at all when there are more than half as many tiles as SMs).  Measured on the LLaDA layer shapes
+// the second choice is as fast or faster at every row count from 2 to 128, so it is the default.
+inline int stream_grid(const UmmaState& st, int n_tiles, int M) {
+  if (st.target_ctas > 0) return st.target_ctas;
+  const int aligned = n_tiles <= st.n_sm ? n_tiles * (st.n_sm / n_tiles) : st.n_sm;
+  if (st.stream_grid_mode == 1) return st.n_sm;
+  if (st.stream_grid_mode == 2) return aligned;
+  return M <= st.stream_even_max_rows ? st.n_sm : aligned;
+}
+
+template <int BN, typename Epi>
+int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
+                  int n_rows_w, const Epi& epi, unsigned* status) {
+  int a_rows = 8;
+  while (a_rows < M) a_rows *= 2;
+  const int stage = 2 * (a_rows * 128 + BN * 128);
+  const int aux = 1024 + 16384 + 8 * (2 * ST_MAX_STAGES + 4) + 16;
+  int stages = (st.max_smem - aux) / stage;
+  if (stages > ST_MAX_STAGES) stages = ST_MAX_STAGES;
+  if (stages > st.max_stages) stages = st.max_stages;
+  if (stages < 2) { st.err = "not enough shared memory for the streaming GEMM"; return -2; }
+  const size_t smem = (size_t)stages * stage + aux;
+  static bool attr_set = false;   // per instantiation
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_stream<BN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, st.max_smem);
+    if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -3; }
+    attr_set = true;
+  }
+  if (st.cache.size() > 4096) st.cache.clear();
+  const CUtensorMap* ma = umma_map(st, A, M, K, a_rows);
+  const CUtensorMap* mb0 = umma_map(st, W0, n_rows_w, K, BN / 2);
+  const CUtensorMap* mb1 = umma_map(st, W1, n_rows_w, K, BN / 2);
+  if (!ma || !mb0 || !mb1) return -4;
+  const int per_tile = Epi::kDual ? BN / 2 : BN;
+  const int n_tiles = (NP + per_tile - 1) / per_tile;
+  const int kc = K / ST_BK;
+  long U = (long)n_tiles * kc;
+  int grid = stream_grid(st, n_tiles, M);
+  if (grid > U) grid = (int)U;
+  StreamArgs args{M, NP, n_tiles, kc, a_rows, stages, st.scratch, st.counters, status};
+  k_gemm_stream<BN, Epi><<<grid, UM_THREADS, smem, stream>>>(*ma, *mb0, *mb1, args, epi);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
+  return 0;
+}
+
+// True when the streaming kernel can take the problem: one row tile, K in whole 128-element chunks, and scratch and
+// counters large enough for its grid.
+template <typename Epi>
+bool stream_eligible(const UmmaState& st, int M, int NP, int K, int bn) {
+  if (!st.use_stream || M > UM_BM || K % ST_BK || st.scratch == nullptr) return false;
+  const int per_tile = Epi::kDual ? bn / 2 : bn;
+  const int n_tiles = (NP + per_tile - 1) / per_tile;
+  return n_tiles <= st.n_counters && stream_scratch_bytes(stream_grid(st, n_tiles, M), bn) <= st.scratch_bytes;
+}
+
+}  // namespace lsp

@@ -202,6 +202,8 @@ struct UmmaArgs {
   int K;
   int num_kb;   // K / 64
   int stages;
+  int a_rows;   // rows of the activation box (8..128): a single-tile launch loads only the rows that exist (rounded up);
+                // accumulator rows beyond them are computed from whatever the stage holds and are never stored
   int m_fast;   // 1: blockIdx.x walks the row tiles (keeps one weight tile hot in L2 across the rows), 0: the column tiles
   int splits;        // split-K factor (blockIdx.z); 1 = none
   int kb_per_split;  // k-blocks per split (the last split may get fewer)
@@ -211,7 +213,7 @@ struct UmmaArgs {
 };
 
 template <int BN>
-constexpr int umma_stage_bytes() { return UM_BM * UM_BK * 2 + BN * UM_BK * 2; }
+constexpr int umma_stage_bytes() { return UM_BM * UM_BK * 2 + BN * UM_BK * 2; }   // with a full activation tile
 
 // Split-K epilogue: publishes this CTA's partial tile; the CTA that arrives last at the tile sums all partials in
 // split order (deterministic) and runs the fused epilogue.  Returns false when the launch is not split.
@@ -291,10 +293,10 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
 k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
             const __grid_constant__ CUtensorMap map_b1, UmmaArgs args, Epi epi) {
   extern __shared__ uint8_t smem_raw[];
-  constexpr int A_BYTES = UM_BM * UM_BK * 2;
   constexpr int B_HALF_BYTES = (BN / 2) * UM_BK * 2;
-  constexpr int STAGE_BYTES = A_BYTES + 2 * B_HALF_BYTES;
   constexpr int HALF = BN / 2;
+  const int A_BYTES = args.a_rows * UM_BK * 2;             // a multiple of 1024: the weight tile stays swizzle-aligned
+  const int STAGE_BYTES = A_BYTES + 2 * B_HALF_BYTES;
   // 1024-byte alignment for the swizzled tiles
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int S = args.stages;
@@ -473,6 +475,13 @@ struct UmmaState {
   int target_ctas = 0;             // 0 = one CTA per SM
   int max_stages = UM_MAX_STAGES;
   int allow_split = 1;
+  int sm_smem = 233472;            // shared memory per SM
+  int skinny_ctas_per_sm = 2;      // co-resident CTAs a weight-streaming (M <= 128) launch aims for
+  int skinny_min_stages = 3;       // ... provided each still gets this many pipeline stages
+  int skinny_bn = 128;             // tile width of plain epilogues in that regime
+  int use_stream = 1;              // M <= 128: use the persistent weight-streaming kernel (gemm_stream.cuh)
+  int stream_grid_mode = 2;        // its grid: 0 = by row count, 1 = one CTA per SM (even shares), 2 = multiple of the tile count
+  int stream_even_max_rows = 0;    // mode 0: even shares up to this many activation rows
   std::string err;
 };
 
@@ -489,6 +498,7 @@ inline int umma_init(UmmaState& st) {
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&st.max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
   cudaDeviceGetAttribute(&st.n_sm, cudaDevAttrMultiProcessorCount, dev);
+  cudaDeviceGetAttribute(&st.sm_smem, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
   return 0;
 }
 
@@ -515,13 +525,25 @@ inline const CUtensorMap* umma_map(UmmaState& st, const void* base, int rows, in
 constexpr int UM_HEAD_BN = 256;
 inline int umma_head_tiles(int vocab) { return (vocab + UM_HEAD_BN - 1) / UM_HEAD_BN; }
 
+// Launch shape of one GEMM, chosen by umma_gemm.
+struct UmmaPlan {
+  int splits = 1;        // split-K factor
+  int a_rows = UM_BM;    // rows of the activation box
+  int smem_cap = 0;      // dynamic shared memory the CTA may use (0 = the device maximum): a lower cap lets two CTAs share an SM
+};
+
 template <int BN, typename Epi>
 int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
-                int n_rows_w, const Epi& epi, unsigned* status, int splits) {
-  constexpr int stage = umma_stage_bytes<BN>();
-  const int aux = 1024 /*alignment slack*/ + 8 * (2 * UM_MAX_STAGES + 1) + 16;
-  int stages = (st.max_smem - aux) / stage;
+                int n_rows_w, const Epi& epi, unsigned* status, UmmaPlan plan) {
+  const int stage = plan.a_rows * UM_BK * 2 + BN * UM_BK * 2;
+  // the MMA always reads 128 activation rows from the stage: rows past the box come from the rest of the stage (or, for
+  // narrow tiles, from the padding appended here) and only feed accumulator rows that are never stored
+  const int pad = stage < UM_BM * UM_BK * 2 ? UM_BM * UM_BK * 2 - stage : 0;
+  const int aux = 1024 /*alignment slack*/ + 8 * (2 * UM_MAX_STAGES + 1) + 16 + pad;
+  const int cap = plan.smem_cap > 0 && plan.smem_cap < st.max_smem ? plan.smem_cap : st.max_smem;
+  int stages = (cap - aux) / stage;
   if (stages > st.max_stages) stages = st.max_stages;
+  int splits = plan.splits;
   const int num_kb = K / UM_BK;
   const int kb_per_split = (num_kb + splits - 1) / splits;
   splits = (num_kb + kb_per_split - 1) / kb_per_split;      // no empty split
@@ -535,7 +557,7 @@ int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W
     attr_set = true;
   }
   if (st.cache.size() > 4096) st.cache.clear();
-  const CUtensorMap* ma = umma_map(st, A, M, K, UM_BM);
+  const CUtensorMap* ma = umma_map(st, A, M, K, plan.a_rows);
   const CUtensorMap* mb0 = umma_map(st, W0, n_rows_w, K, BN / 2);
   const CUtensorMap* mb1 = umma_map(st, W1, n_rows_w, K, BN / 2);
   if (!ma || !mb0 || !mb1) return -4;
@@ -544,49 +566,93 @@ int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W
   dim3 grid((NP + per_tile - 1) / per_tile, (M + UM_BM - 1) / UM_BM);
   if (m_fast) grid = dim3(grid.y, grid.x);
   grid.z = splits;
-  UmmaArgs args{M, NP, K, num_kb, stages, m_fast, splits, kb_per_split, st.scratch, st.counters, status};
+  UmmaArgs args{M, NP, K, num_kb, stages, plan.a_rows, m_fast, splits, kb_per_split, st.scratch, st.counters, status};
   k_gemm_umma<BN, Epi><<<grid, UM_THREADS, smem, stream>>>(*ma, *mb0, *mb1, args, epi);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
   return 0;
 }
 
-// Tile-width and split-K choice.  Large problems (at least one CTA per SM without splitting) take the widest tile.
-// Small-M problems are bound by streaming the weights once: they take 128-column tiles (so the activation tile is not
-// re-read more often than the weights) and split K until every SM has a CTA.  The rotary epilogue needs both partners
-// of a pair inside one head, which caps the tile at head_dim columns.
+template <typename Epi> bool stream_eligible(const UmmaState& st, int M, int NP, int K, int bn);
+template <int BN, typename Epi>
+int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
+                  int n_rows_w, const Epi& epi, unsigned* status);
+
+// Tile-width and split-K choice.
+//  * Problems with at most 128 activation rows go to the persistent weight-streaming kernel (gemm_stream.cuh) when it
+//    is eligible; the rules below cover the rest.
+//  * Large problems (at least one CTA per SM without splitting) take the widest tile, one CTA per SM, deepest pipeline.
+//  * Single-row-tile problems (M <= 128) are bound by streaming the weights from HBM once.  Measured on B200, one
+//    CTA per SM that fetches 128 bytes per weight row per stage tops out near 3.7 TB/s however deep its pipeline is,
+//    while two co-resident CTAs per SM (or 256 bytes per row per stage) reach 5.3 TB/s.  So these launches load only
+//    the activation rows that exist (a box of 8..128 rows), cap their shared memory at half an SM so that two CTAs
+//    fit, and split K until both CTA slots of every SM are filled in a single wave.
+//  * The rotary epilogue needs both partners of a pair inside one head, which caps its tile at head_dim columns.
 template <typename Epi>
 int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
               int n_rows_w, const Epi& epi, unsigned* status) {
   if (K % UM_BK) { st.err = "K must be a multiple of 64"; return -6; }
+  const int mt = (M + UM_BM - 1) / UM_BM;
+  UmmaPlan plan;
+  if (mt == 1) {
+    plan.a_rows = 8;
+    while (plan.a_rows < M) plan.a_rows *= 2;
+  }
   if constexpr (Epi::kReduce) {
-    return umma_launch<UM_HEAD_BN, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 1);
+    if (stream_eligible<Epi>(st, M, NP, K, UM_HEAD_BN))
+      return stream_launch<UM_HEAD_BN, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+    if (mt == 1 && st.skinny_ctas_per_sm > 1) {
+      const int stage = plan.a_rows * UM_BK * 2 + UM_HEAD_BN * UM_BK * 2;
+      const int cap = (st.sm_smem / 2 - 1024) & ~1023;       // 2 x 256 accumulator columns fill the tensor memory
+      if ((cap - 2048) / stage >= st.skinny_min_stages) plan.smem_cap = cap;
+    }
+    return umma_launch<UM_HEAD_BN, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
   } else {
     const int cols = Epi::kDual ? 2 * NP : NP;
-    const int mt = (M + UM_BM - 1) / UM_BM;
     const int num_kb = K / UM_BK;
     int max_bn = 256;
     if constexpr (std::is_same<Epi, EpiQKVRope<bf16>>::value) max_bn = 2 * epi.half;
-    const int target = st.target_ctas > 0 ? st.target_ctas : st.n_sm;
-    int bn = max_bn, splits = 1;
+    {
+      const int sbn = Epi::kDual ? max_bn : (max_bn < 128 ? max_bn : 128);
+      if (stream_eligible<Epi>(st, M, NP, K, sbn)) {
+        switch (sbn) {
+          case 256: return stream_launch<256, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+          case 128: return stream_launch<128, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+          case 64: return stream_launch<64, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+          default: break;
+        }
+      }
+    }
+    int bn = max_bn;
     const long big_tiles = (long)mt * ((cols + max_bn - 1) / max_bn);
-    if (big_tiles < target) {
-      bn = Epi::kDual ? max_bn : (max_bn < 128 ? max_bn : 128);
+    if (big_tiles < st.n_sm) {
+      bn = Epi::kDual ? max_bn : (max_bn < st.skinny_bn ? max_bn : st.skinny_bn);
       const long tiles = (long)mt * ((cols + bn - 1) / bn);
-      if (st.allow_split && st.scratch != nullptr && tiles < target) {
-        splits = (int)((target + tiles / 2) / tiles);
+      int slots = st.n_sm;
+      if (mt == 1 && st.skinny_ctas_per_sm > 1) {
+        const int stage = plan.a_rows * UM_BK * 2 + bn * UM_BK * 2;
+        const int cap = (st.sm_smem / st.skinny_ctas_per_sm - 1024) & ~1023;
+        if ((cap - 2048) / stage >= st.skinny_min_stages) {
+          plan.smem_cap = cap;
+          slots = st.n_sm * st.skinny_ctas_per_sm;
+        }
+      }
+      if (st.target_ctas > 0) slots = st.target_ctas;
+      if (st.allow_split && st.scratch != nullptr && tiles < slots) {
+        int splits = (int)(slots / tiles);
         if (splits > num_kb / 4) splits = num_kb / 4;
         if (splits < 1) splits = 1;
         while (splits > 1 && ((size_t)tiles * splits * UM_BM * bn * sizeof(float) > st.scratch_bytes ||
                               tiles > st.n_counters))
           --splits;
+        plan.splits = splits;
       }
     }
     switch (bn) {
-      case 256: return umma_launch<256, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, splits);
-      case 128: return umma_launch<128, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, splits);
-      case 64: return umma_launch<64, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, splits);
-      default: return umma_launch<32, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, splits);
+      case 256: return umma_launch<256, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
+      case 128: return umma_launch<128, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
+      case 64: return umma_launch<64, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
+      default: return umma_launch<32, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
     }
   }
 }

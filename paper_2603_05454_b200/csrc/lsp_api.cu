@@ -15,7 +15,7 @@
 #include "gemm_simt.cuh"
 #include "misc_kernels.cuh"
 #ifndef LSP_NO_UMMA
-#include "gemm_umma.cuh"
+#include "gemm_stream.cuh"
 #endif
 
 using namespace lsp;
@@ -616,6 +616,12 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   else if (key == 10) c->umma.target_ctas = value;
   else if (key == 11) c->umma.max_stages = value < 1 ? 1 : (value > UM_MAX_STAGES ? UM_MAX_STAGES : value);
   else if (key == 12) c->umma.allow_split = value;
+  else if (key == 16) c->umma.use_stream = value;
+  else if (key == 17) c->umma.stream_grid_mode = value;
+  else if (key == 18) c->umma.stream_even_max_rows = value;
+  else if (key == 13) c->umma.skinny_ctas_per_sm = value < 1 ? 1 : value;
+  else if (key == 14) c->umma.skinny_min_stages = value < 1 ? 1 : value;
+  else if (key == 15) c->umma.skinny_bn = (value == 64 || value == 32) ? value : 128;
 #endif
   else return fail(c, LSP_ERR_ARG, "lsp_set_option: unknown key %d", key);
   return LSP_OK;

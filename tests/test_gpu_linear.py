@@ -53,3 +53,39 @@ def test_linear_fp32(shape):
                                    (512, 4096, 4096), (37, 12288, 4096), (257, 4096, 12288)])
 def test_linear_bf16(impl, shape):
     _check("bf16", impl, *shape, seed=1)
+
+
+@pytest.mark.parametrize("grid_mode", [1, 2])
+@pytest.mark.parametrize("shape", [(1, 256, 128), (5, 384, 256), (64, 1152, 512), (128, 4096, 4096), (100, 12288, 4096),
+                                   (17, 4096, 12288)])
+def test_linear_bf16_weight_streaming_kernel(grid_mode, shape):
+    """M <= 128 and K in whole 128-element chunks take the persistent streaming kernel: tiles split between CTAs
+    (partials in scratch, summed by the last arriver) with both ways of dealing out the work."""
+    M, N, K = shape
+    tdt = torch.bfloat16
+    dec = _dec("bf16")
+    dec.set_option(17, grid_mode)
+    A = S.normal((M, K), 2, 1, 1.0, tdt, DEV)
+    W = S.normal((N, K), 2, 2, 0.05, tdt, DEV)
+    W2 = S.normal((N, K), 2, 3, 0.05, tdt, DEV)
+    X0 = S.normal((M, N), 2, 4, 1.0, tdt, DEV)
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    a, w, w2, x0 = f64(A), f64(W), f64(W2), f64(X0)
+    rtol = 1.0 / 128
+    out = torch.empty(M, N, dtype=tdt, device=DEV)
+    outs = []
+    for rep in range(2):                       # twice: the tile counters must be back at zero after a launch
+        dec.op_linear(0, A, W, None, out)
+        ref = a @ w.T
+        np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05)
+        outs.append(out.clone())
+    assert torch.equal(outs[0], outs[1])       # deterministic summation order
+    xr = X0.clone()
+    dec.op_linear(1, A, W, None, xr)
+    ref = x0 + a @ w.T
+    np.testing.assert_allclose(f64(xr), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05)
+    dec.op_linear(2, A, W, W2, out)
+    g, u = a @ w.T, a @ w2.T
+    ref = g / (1 + np.exp(-g)) * u
+    np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05)
+    dec.close()
