@@ -130,7 +130,10 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * 14 = fewest pipeline stages it accepts for that, 15 = its tile width for plain epilogues (32, 64 or 128),
  * 16 = GEMMs with at most 128 rows use the persistent weight-streaming kernel (1, default) or the tiled one (0),
  * 17 = grid of that kernel (0 by row count, 1 one CTA per SM with even shares, 2 a multiple of the tile count),
- * 18 = row count up to which mode 0 takes even shares. */
+ * 18 = row count up to which mode 0 takes even shares, 19 = that kernel also takes 129..256 rows (1, default) or not (0),
+ * 20 = its tile width for those (0 = automatic, 64, 128 or 256), 21 = 64-element K atoms per pipeline stage (0 = automatic, 1, 2),
+ * 22 = fewest two-atom stages the automatic choice accepts, 23 = its tile width for up to 128 rows (0 = automatic,
+ * 64, 128 or 256). */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

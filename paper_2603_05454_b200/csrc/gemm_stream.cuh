@@ -1,20 +1,26 @@
-// Weight-streaming bf16 GEMM for at most 128 activation rows (the shrinking suffix of late decode steps), tcgen05.
+// Weight-streaming bf16 GEMM for at most 256 activation rows (the shrinking suffix of late decode steps), tcgen05.
 //
 //   acc[m, c] = sum_k A[m, k] * Wt[c, k]        same operands, tiles and fused epilogues as gemm_umma.cuh
 //
-// With M <= 128 a layer GEMM is bound by reading its weights from HBM once, so the kernel is built around one
-// uninterrupted stream of weight tiles per SM:
+// With M <= 256 a layer GEMM is bound by reading its weights from HBM once (at the upper end the tensor cores need
+// about as long), so the kernel is built around one uninterrupted stream of weight tiles per SM, each weight tile
+// being used for every activation row while it is in shared memory (MT = 1 or 2 row tiles of 128, one accumulator
+// each):
 //   * persistent CTAs, at most one per SM; the (column tile, K chunk) units of the whole problem are dealt out in
 //     equal contiguous shares (a share may start and end in the middle of a tile), in a single wave;
-//   * a pipeline stage holds 128 elements of K (two 128-byte swizzle atoms per operand): 256 contiguous bytes per
-//     weight row and stage, which on B200 streams at 5.3 TB/s where 128 bytes per row and stage reach only 3.7 TB/s;
-//   * only the activation rows that exist are loaded (a box of 8..128 rows); the MMA still spans 128 accumulator rows,
-//     and the rows past the box, computed from whatever the stage holds, are never stored;
-//   * accumulators are double-buffered in tensor memory, so the epilogue of one tile overlaps the loads and MMAs of
-//     the next; only the first fill and the last epilogue of a CTA are exposed;
+//   * a pipeline stage holds 128 elements of K (two 128-byte swizzle atoms per operand) when at least three such
+//     stages fit, else 64: 256 contiguous bytes per weight row and stage stream at 5.3 TB/s on B200 where 128 bytes
+//     per row and stage reach only 3.7 TB/s;
+//   * only the activation rows that exist are loaded (a box of M rounded up to 8 rows); the MMAs still span 128
+//     accumulator rows each, and the rows past the box, computed from whatever the stage holds, are never stored;
+//   * accumulators are double-buffered in tensor memory when two sets fit in its 512 columns, so the epilogue of one
+//     tile overlaps the loads and MMAs of the next; only the first fill and the last epilogue of a CTA are exposed;
 //   * a tile that spans several CTAs is finished by the CTA that arrives last at the tile's counter: every
 //     contributor writes its fp32 partial tile to scratch, and the finisher sums all of them in CTA order (the same
 //     order whoever finishes, so results are deterministic) before running the fused epilogue.
+// Tile width: one tcgen05.mma with M = 128 occupies the tensor pipe for about 150 cycles whatever its N (measured
+// for N = 16..256), so a narrow tile does not make the instruction cheaper; 256-column tiles halve the instruction
+// count per weight byte against 128-column ones and keep the MMA time below the weight-streaming time.
 // Warp roles as in gemm_umma.cuh: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = epilogue.
 // Every wait is bounded; on expiry the kernel records (code, site) in the status word, drains and returns.
 #pragma once
@@ -22,17 +28,18 @@
 
 namespace lsp {
 
-constexpr int ST_BK = 128;                 // K elements per stage (two swizzle atoms)
 constexpr int ST_MAX_STAGES = 8;
 
 struct StreamArgs {
-  int M;            // activation rows (<= 128)
+  int M;            // activation rows (<= 128 MT)
   int n_pairs;      // dual: pair indices; plain: output columns
   int n_tiles;      // column tiles
-  int kc;           // K / 128 chunks per tile
-  int a_rows;       // activation box rows (8..128, power of two)
+  int kc;           // K chunks (one per stage) per tile
+  int a_rows;       // activation box rows (M rounded up to a multiple of 8)
+  int atoms;        // 64-element K atoms per stage (1 or 2)
+  int box_rows;     // weight rows per TMA box: BN/2, or fewer when the rows of a half tile are not contiguous (rotary pairs)
   int stages;
-  float* scratch;   // [gridDim.x][2][128][BN] fp32 partial tiles
+  float* scratch;   // [gridDim.x][2][128 MT][BN] fp32 partial tiles
   unsigned* counters;  // one per column tile, zero between launches
   unsigned* status;
 };
@@ -46,7 +53,7 @@ __device__ __forceinline__ long st_first_unit(long U, int G, int g) { return U *
 // CTA that owns unit u
 __device__ __forceinline__ int st_owner(long U, int G, long u) { return (int)(((u + 1) * G + U - 1) / U) - 1; }
 
-template <int BN, typename Epi>
+template <int BN, int MT, typename Epi>
 __global__ void __launch_bounds__(UM_THREADS, 1)
 k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
               const __grid_constant__ CUtensorMap map_b1, StreamArgs args, Epi epi) {
@@ -54,12 +61,16 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   constexpr int HALF = BN / 2;
   constexpr int B_HALF_ATOM = HALF * 128;               // bytes of one half-tile atom (64 K elements)
   constexpr int B_ATOM = BN * 128;
+  constexpr int ROWS = UM_BM * MT;                        // accumulator rows
+  constexpr int NBUF = (2 * MT * BN <= 512) ? 2 : 1;      // accumulator sets in tensor memory
+  constexpr uint32_t TMEM_COLS = NBUF * MT * BN;
   const int A_ATOM = args.a_rows * 128;
-  const int STAGE_BYTES = 2 * (A_ATOM + B_ATOM);
+  const int AT = args.atoms;
+  const int STAGE_BYTES = AT * (A_ATOM + B_ATOM);
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int S = args.stages;
-  // the barriers sit behind the stages and 16 KB of padding the MMA may read (never written) past the last stage
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * STAGE_BYTES + 16384);
+  // the barriers sit behind the stages and the padding the MMA may read (never written) past the last stage
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * STAGE_BYTES + ROWS * 128);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) accumulator full, [2S+2..2S+4) accumulator empty
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 4);
   volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -87,7 +98,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"((uint32_t)(2 * BN))
+                 "r"(TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -112,20 +123,20 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
           break;
         }
         const int tile = (int)(u / args.kc), c = (int)(u % args.kc);
-        int row_b0, row_b1;
-        if (Epi::kDual) { row_b0 = epi.row0(tile * HALF); row_b1 = epi.row1(tile * HALF); }
-        else { row_b0 = tile * BN; row_b1 = tile * BN + HALF; }
         mbar_expect_tx(full_bar(s), STAGE_BYTES);
         const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
-        const uint32_t sb = sa + 2 * A_ATOM;
-        const int k0 = c * ST_BK;
-        // weights first, both atoms of a row group back to back: 256 contiguous bytes per weight row
-        tma_load_2d(sb, &map_b0, k0, row_b0, full_bar(s));
-        tma_load_2d(sb + B_ATOM, &map_b0, k0 + 64, row_b0, full_bar(s));
-        tma_load_2d(sb + B_HALF_ATOM, &map_b1, k0, row_b1, full_bar(s));
-        tma_load_2d(sb + B_ATOM + B_HALF_ATOM, &map_b1, k0 + 64, row_b1, full_bar(s));
-        tma_load_2d(sa, &map_a, k0, 0, full_bar(s));
-        tma_load_2d(sa + A_ATOM, &map_a, k0 + 64, 0, full_bar(s));
+        const uint32_t sb = sa + AT * A_ATOM;
+        const int k0 = c * AT * UM_BK;
+        // weights first, the atoms of a row group back to back: AT x 128 contiguous bytes per weight row
+        for (int b = 0; b < HALF; b += args.box_rows) {
+          int row_b0, row_b1;
+          if (Epi::kDual) { row_b0 = epi.row0(tile * HALF + b); row_b1 = epi.row1(tile * HALF + b); }
+          else { row_b0 = tile * BN + b; row_b1 = tile * BN + HALF + b; }
+          for (int j = 0; j < AT; ++j) tma_load_2d(sb + j * B_ATOM + b * 128, &map_b0, k0 + 64 * j, row_b0, full_bar(s));
+          for (int j = 0; j < AT; ++j)
+            tma_load_2d(sb + j * B_ATOM + B_HALF_ATOM + b * 128, &map_b1, k0 + 64 * j, row_b1, full_bar(s));
+        }
+        for (int j = 0; j < AT; ++j) tma_load_2d(sa + j * A_ATOM, &map_a, k0 + 64 * j, 0, full_bar(s));
         ++issued;
       }
       // do not leave while copies may still be landing in this CTA's shared memory
@@ -144,15 +155,15 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
       for (long u = u0; u < u1 && ok;) {
         const int tile = (int)(u / args.kc);
         const long seg_end = min(u1, (long)(tile + 1) * args.kc);
-        const int buf = seg & 1;
-        // wait until the epilogue has drained this accumulator buffer (its previous use was segment seg - 2)
-        if (seg >= 2 && !mbar_wait(acce_bar(buf), (uint32_t)((seg >> 1) - 1) & 1u, abort_flag)) {
+        const int buf = seg % NBUF, use = seg / NBUF;
+        // wait until the epilogue has drained this accumulator set (its previous use was segment seg - NBUF)
+        if (use >= 1 && !mbar_wait(acce_bar(buf), (uint32_t)(use - 1) & 1u, abort_flag)) {
           if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 12u; }
           ok = false;
           break;
         }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
         bool first = true;
         for (; u < seg_end; ++u) {
           const int it = (int)(u - u0), s = it % S;
@@ -164,14 +175,16 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
           }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
-          const uint32_t sb = sa + 2 * A_ATOM;
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
+          const uint32_t sb = sa + AT * A_ATOM;
+          for (int j = 0; j < AT; ++j) {
             const uint64_t da = make_smem_desc(sa + j * A_ATOM);
             const uint64_t db = make_smem_desc(sb + j * B_ATOM);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              tc_mma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, first ? 0u : 1u);
+#pragma unroll
+              for (int mt = 0; mt < MT; ++mt)   // row tile mt starts 128 rows = 16 KB further into the activation atom
+                tc_mma_f16(d_tmem + (uint32_t)(mt * BN), da + (uint64_t)(mt * 1024 + 2 * k), db + (uint64_t)(2 * k), idesc,
+                           first ? 0u : 1u);
               first = false;
             }
           }
@@ -184,8 +197,8 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   } else {
     // ---------------- epilogue (warps 2..5) ----------------
     const int q = warp & 3;
-    const int r_in = q * 32 + lane;
-    const int m = r_in;
+    const int r_in = q * 32 + lane;                       // accumulator lane this thread reads
+    constexpr int CH = Epi::kDual ? HALF : BN;            // pair indices (dual) or columns (plain) per tile
     int seg = 0;
     bool ok = true;
     for (long u = u0; u < u1 && ok; ++seg) {
@@ -193,31 +206,66 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
       const long tile_u0 = (long)tile * args.kc;
       const long seg_end = min(u1, tile_u0 + args.kc);
       const bool whole = (u == tile_u0) && (seg_end == tile_u0 + args.kc);
-      const int buf = seg & 1;
-      if (!mbar_wait(accf_bar(buf), (uint32_t)(seg >> 1) & 1u, abort_flag)) {
+      const int buf = seg % NBUF, use = seg / NBUF;
+      if (!mbar_wait(accf_bar(buf), (uint32_t)use & 1u, abort_flag)) {
         if (lane == 0 && !*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 14u; }
         ok = false;
         break;
       }
       tc_fence_after();
-      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
-      bool finish = whole;
-      int g_lo = g, g_hi = g;
-      if (!whole) {
-        // publish this CTA's partial tile, then count its chunks in; the CTA that completes the count finishes the tile
-        // partial tile layout: [16-column chunk][quarter][row][4 floats], so that the lanes of a warp (consecutive
-        // rows) write and read consecutive 16-byte pieces
-        float4* mine = reinterpret_cast<float4*>(args.scratch + (size_t)(g * 2 + (seg == 0 ? 0 : 1)) * UM_BM * BN) + r_in;
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * MT * BN);
+      const int j0 = tile * CH;
+      if (whole) {
+        // the accumulator is complete in tensor memory: each thread owns one row of every row tile
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 16) {
-          float v[16];
-          tc_ld16(t_row + c, v);
-          if (m < args.M) {
+        for (int mt = 0; mt < MT; ++mt) {
+          const int m = mt * UM_BM + r_in;
+          Top2 red = top2_empty();
+#pragma unroll 1
+          for (int c = 0; c < CH; c += 16) {
+            float a0[16], a1[16];
+            tc_ld16(t_row + mt * BN + c, a0);
+            if (Epi::kDual) tc_ld16(t_row + mt * BN + HALF + c, a1);
+            if constexpr (Epi::kReduce) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-              mine[(size_t)((c >> 4) * 4 + i) * UM_BM] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+              for (int i = 0; i < 16; ++i) {
+                const int col = j0 + c + i;
+                if (epi.valid(col)) top2_push(red, a0[i], col);
+              }
+            } else {
+              if (m < args.M && j0 + c < args.n_pairs) epi16(epi, m, j0 + c, a0, a1);
+            }
+          }
+          if constexpr (Epi::kReduce) {
+            if (m < args.M) epi.part[(size_t)m * epi.n_tiles + tile] = red;
           }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(buf));
+      } else {
+        // publish this CTA's partial tile, then count its chunks in; the CTA that completes the count finishes the tile.
+        // Partial tile layout: [16-column chunk][quarter][row][4 floats], so that the lanes of a warp (consecutive
+        // rows) write and read consecutive 16-byte pieces.
+        float4* slot_base = reinterpret_cast<float4*>(args.scratch + (size_t)(g * 2 + (seg == 0 ? 0 : 1)) * ROWS * BN);
+#pragma unroll 1
+        for (int mt = 0; mt < MT; ++mt) {
+          const int m = mt * UM_BM + r_in;
+#pragma unroll 1
+          for (int c = 0; c < BN; c += 16) {
+            float v[16];
+            tc_ld16(t_row + mt * BN + c, v);
+            if (m < args.M) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                slot_base[(size_t)((c >> 4) * 4 + i) * ROWS + m] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+          }
+        }
+        // the accumulator set is free as soon as every warp has read it
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(buf));
         __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (threadIdx.x == 64) {
@@ -228,113 +276,75 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
           *epi_flag = last ? 1u : 0u;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        finish = (*epi_flag != 0);
-        if (finish) {
+        if (*epi_flag != 0) {
           __threadfence();
-          g_lo = st_owner(U, G, tile_u0);
-          g_hi = st_owner(U, G, tile_u0 + args.kc - 1);
-        }
-      }
-      // the accumulator buffer is free once every warp has read it (whole tiles read it below)
-      if (!whole) {
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(acce_bar(buf));
-      }
-      constexpr int CH = Epi::kDual ? HALF : BN;   // pair indices (dual) or columns (plain) per tile
-      const int j0 = tile * CH;
-      if (finish && whole) {
-        // the accumulator is complete in tensor memory: each thread owns one row
-        Top2 red = top2_empty();
-#pragma unroll 1
-        for (int c = 0; c < CH; c += 16) {
-          float a0[16], a1[16];
-          tc_ld16(t_row + c, a0);
-          if (Epi::kDual) tc_ld16(t_row + HALF + c, a1);
-          if constexpr (Epi::kReduce) {
+          const int g_lo = st_owner(U, G, tile_u0), g_hi = st_owner(U, G, tile_u0 + args.kc - 1);
+          // The tile is the sum of the contributors' partial tiles.  Work items are (row, 16-column chunk), dealt over
+          // the 128 epilogue threads so that a tile with few rows still uses all of them, and every item issues the
+          // loads of up to four contributors before it adds them (in CTA order: deterministic).
+          constexpr int NCH = CH / 16;                 // chunks per row
+          constexpr int RPP = 128 / NCH;               // rows per pass
+          const int et = threadIdx.x - 64;
+          // plain epilogues: consecutive lanes take consecutive rows (coalesced reads of the partials); the reducing
+          // epilogue keeps a row's chunks in neighbouring lanes so that they can be merged with shuffles
+          const int ch = Epi::kReduce ? et % NCH : et / RPP, c = ch * 16;
+          for (int mm0 = 0; mm0 < args.M; mm0 += RPP) {
+            const int mm = mm0 + (Epi::kReduce ? et / NCH : et % RPP);
+            const bool valid = mm < args.M;
+            float a0[16], a1[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const int col = j0 + c + i;
-              if (epi.valid(col)) top2_push(red, a0[i], col);
-            }
-          } else {
-            if (m < args.M && j0 + c < args.n_pairs) epi16(epi, m, j0 + c, a0, a1);
-          }
-        }
-        if constexpr (Epi::kReduce) {
-          if (m < args.M) epi.part[(size_t)m * epi.n_tiles + tile] = red;
-        }
-      } else if (finish) {
-        // the tile is the sum of the contributors' partial tiles in scratch.  Work items are (row, 16-column chunk),
-        // dealt over the 128 epilogue threads so that a tile with few rows still uses all of them, and every item
-        // issues the loads of up to four contributors before it adds them (in CTA order: deterministic).
-        constexpr int NCH = CH / 16;                 // chunks per row
-        constexpr int RPP = 128 / NCH;               // rows per pass
-        const int et = threadIdx.x - 64;
-        // plain epilogues: consecutive lanes take consecutive rows (coalesced reads of the partials); the reducing
-        // epilogue keeps a row's chunks in neighbouring lanes so that they can be merged with shuffles
-        const int ch = Epi::kReduce ? et % NCH : et / RPP, c = ch * 16;
-        for (int mm0 = 0; mm0 < args.M; mm0 += RPP) {
-          const int mm = mm0 + (Epi::kReduce ? et / NCH : et % RPP);
-          const bool valid = mm < args.M;
-          float a0[16], a1[16];
+            for (int i = 0; i < 16; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
+            if (valid) {
+              for (int gb = g_lo; gb <= g_hi; gb += 4) {
+                float4 t0[4][4], t1[4][4];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
-          if (valid) {
-            for (int gb = g_lo; gb <= g_hi; gb += 4) {
-              float4 t0[4][4], t1[4][4];
+                for (int x = 0; x < 4; ++x) {
+                  const int gg = gb + x;
+                  if (gg <= g_hi) {
+                    // contributor gg's segment of this tile is its first one iff its share starts inside the tile
+                    const int slot = (st_first_unit(U, G, gg) >= tile_u0) ? 0 : 1;
+                    const float4* base = reinterpret_cast<const float4*>(args.scratch + (size_t)(gg * 2 + slot) * ROWS * BN) + mm;
+                    const float4* p0 = base + (size_t)(c >> 4) * 4 * ROWS;
 #pragma unroll
-              for (int x = 0; x < 4; ++x) {
-                const int gg = gb + x;
-                if (gg <= g_hi) {
-                  // contributor gg's segment of this tile is its first one iff its share starts inside the tile
-                  const int slot = (st_first_unit(U, G, gg) >= tile_u0) ? 0 : 1;
-                  const float4* base = reinterpret_cast<const float4*>(args.scratch + (size_t)(gg * 2 + slot) * UM_BM * BN) + mm;
-                  const float4* p0 = base + (size_t)(c >> 4) * 4 * UM_BM;
+                    for (int i = 0; i < 4; ++i) t0[x][i] = __ldcg(p0 + (size_t)i * ROWS);
+                    if (Epi::kDual) {
+                      const float4* p1 = base + (size_t)((HALF + c) >> 4) * 4 * ROWS;
 #pragma unroll
-                  for (int i = 0; i < 4; ++i) t0[x][i] = __ldcg(p0 + (size_t)i * UM_BM);
-                  if (Epi::kDual) {
-                    const float4* p1 = base + (size_t)((HALF + c) >> 4) * 4 * UM_BM;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) t1[x][i] = __ldcg(p1 + (size_t)i * UM_BM);
+                      for (int i = 0; i < 4; ++i) t1[x][i] = __ldcg(p1 + (size_t)i * ROWS);
+                    }
                   }
                 }
-              }
 #pragma unroll
-              for (int x = 0; x < 4; ++x) {
-                if (gb + x <= g_hi) {
+                for (int x = 0; x < 4; ++x) {
+                  if (gb + x <= g_hi) {
 #pragma unroll
-                  for (int i = 0; i < 4; ++i) {
-                    a0[4 * i] += t0[x][i].x; a0[4 * i + 1] += t0[x][i].y; a0[4 * i + 2] += t0[x][i].z; a0[4 * i + 3] += t0[x][i].w;
-                    if (Epi::kDual) {
-                      a1[4 * i] += t1[x][i].x; a1[4 * i + 1] += t1[x][i].y; a1[4 * i + 2] += t1[x][i].z; a1[4 * i + 3] += t1[x][i].w;
+                    for (int i = 0; i < 4; ++i) {
+                      a0[4 * i] += t0[x][i].x; a0[4 * i + 1] += t0[x][i].y; a0[4 * i + 2] += t0[x][i].z; a0[4 * i + 3] += t0[x][i].w;
+                      if (Epi::kDual) {
+                        a1[4 * i] += t1[x][i].x; a1[4 * i + 1] += t1[x][i].y; a1[4 * i + 2] += t1[x][i].z; a1[4 * i + 3] += t1[x][i].w;
+                      }
                     }
                   }
                 }
               }
             }
-          }
-          if constexpr (Epi::kReduce) {
-            Top2 red = top2_empty();
-            if (valid) {
+            if constexpr (Epi::kReduce) {
+              Top2 red = top2_empty();
+              if (valid) {
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const int col = j0 + c + i;
-                if (epi.valid(col)) top2_push(red, a0[i], col);
+                for (int i = 0; i < 16; ++i) {
+                  const int col = j0 + c + i;
+                  if (epi.valid(col)) top2_push(red, a0[i], col);
+                }
               }
-            }
 #pragma unroll
-            for (int o = 1; o < NCH; o <<= 1) red = top2_merge(red, top2_shfl_xor(red, o));
-            if (valid && ch == 0) epi.part[(size_t)mm * epi.n_tiles + tile] = red;
-          } else {
-            if (valid && j0 + c < args.n_pairs) epi16(epi, mm, j0 + c, a0, a1);
+              for (int o = 1; o < NCH; o <<= 1) red = top2_merge(red, top2_shfl_xor(red, o));
+              if (valid && ch == 0) epi.part[(size_t)mm * epi.n_tiles + tile] = red;
+            } else {
+              if (valid && j0 + c < args.n_pairs) epi16(epi, mm, j0 + c, a0, a1);
+            }
           }
         }
-      }
-      if (whole) {
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(acce_bar(buf));
       }
       u = seg_end;
     }
@@ -343,13 +353,13 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(2 * BN)) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
 // ---- host side ------------------------------------------------------------------------------------------------
-// Scratch the streaming kernel needs for a grid of n_ctas CTAs and tile width bn.
-inline size_t stream_scratch_bytes(int n_ctas, int bn) { return (size_t)n_ctas * 2 * UM_BM * bn * sizeof(float); }
+// Scratch the streaming kernel needs for a grid of n_ctas CTAs, tile width bn and mt row tiles.
+inline size_t stream_scratch_bytes(int n_ctas, int bn, int mt) { return (size_t)n_ctas * 2 * UM_BM * mt * bn * sizeof(float); }
 
 // Number of CTAs.  Dealing the units evenly over all SMs balances the weight stream perfectly but splits almost every
 // tile between two CTAs, which costs a partial tile written and read back per split (M x BN x 4 bytes each way).
@@ -364,50 +374,64 @@ inline int stream_grid(const UmmaState& st, int n_tiles, int M) {
   return M <= st.stream_even_max_rows ? st.n_sm : aligned;
 }
 
-template <int BN, typename Epi>
+// Stage shape for M rows and tile width bn: two K atoms per stage when at least three such stages fit.
+struct StreamShape { int a_rows, atoms, stages, stage_bytes, aux; };
+inline StreamShape stream_shape(const UmmaState& st, int M, int bn, int mt, int K) {
+  StreamShape sh;
+  sh.a_rows = (M + 7) / 8 * 8;
+  sh.aux = 1024 + UM_BM * mt * 128 + 8 * (2 * ST_MAX_STAGES + 4) + 16;
+  const int atom = sh.a_rows * 128 + bn * 128;
+  sh.atoms = (K % 128 == 0 && (st.max_smem - sh.aux) / (2 * atom) >= st.stream_min_stages2) ? 2 : 1;
+  if (st.stream_atoms == 1 || (st.stream_atoms == 2 && K % 128 == 0)) sh.atoms = st.stream_atoms;
+  sh.stage_bytes = sh.atoms * atom;
+  sh.stages = (st.max_smem - sh.aux) / sh.stage_bytes;
+  if (sh.stages > ST_MAX_STAGES) sh.stages = ST_MAX_STAGES;
+  if (sh.stages > st.max_stages) sh.stages = st.max_stages;
+  return sh;
+}
+
+template <int BN, int MT, typename Epi>
 int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
-                  int n_rows_w, const Epi& epi, unsigned* status) {
-  int a_rows = 8;
-  while (a_rows < M) a_rows *= 2;
-  const int stage = 2 * (a_rows * 128 + BN * 128);
-  const int aux = 1024 + 16384 + 8 * (2 * ST_MAX_STAGES + 4) + 16;
-  int stages = (st.max_smem - aux) / stage;
-  if (stages > ST_MAX_STAGES) stages = ST_MAX_STAGES;
-  if (stages > st.max_stages) stages = st.max_stages;
-  if (stages < 2) { st.err = "not enough shared memory for the streaming GEMM"; return -2; }
-  const size_t smem = (size_t)stages * stage + aux;
+                  int n_rows_w, const Epi& epi, unsigned* status, int box_rows) {
+  const StreamShape sh = stream_shape(st, M, BN, MT, K);
+  if (sh.stages < 2) { st.err = "not enough shared memory for the streaming GEMM"; return -2; }
+  const size_t smem = (size_t)sh.stages * sh.stage_bytes + sh.aux;
   static bool attr_set = false;   // per instantiation
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(k_gemm_stream<BN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, st.max_smem);
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_stream<BN, MT, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, st.max_smem);
     if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -3; }
     attr_set = true;
   }
   if (st.cache.size() > 4096) st.cache.clear();
-  const CUtensorMap* ma = umma_map(st, A, M, K, a_rows);
-  const CUtensorMap* mb0 = umma_map(st, W0, n_rows_w, K, BN / 2);
-  const CUtensorMap* mb1 = umma_map(st, W1, n_rows_w, K, BN / 2);
+  const CUtensorMap* ma = umma_map(st, A, M, K, sh.a_rows);
+  if (box_rows <= 0 || box_rows > BN / 2 || (BN / 2) % box_rows || box_rows % 8) box_rows = BN / 2;
+  const CUtensorMap* mb0 = umma_map(st, W0, n_rows_w, K, box_rows);
+  const CUtensorMap* mb1 = umma_map(st, W1, n_rows_w, K, box_rows);
   if (!ma || !mb0 || !mb1) return -4;
   const int per_tile = Epi::kDual ? BN / 2 : BN;
   const int n_tiles = (NP + per_tile - 1) / per_tile;
-  const int kc = K / ST_BK;
+  const int kc = K / (sh.atoms * UM_BK);
   long U = (long)n_tiles * kc;
   int grid = stream_grid(st, n_tiles, M);
   if (grid > U) grid = (int)U;
-  StreamArgs args{M, NP, n_tiles, kc, a_rows, stages, st.scratch, st.counters, status};
-  k_gemm_stream<BN, Epi><<<grid, UM_THREADS, smem, stream>>>(*ma, *mb0, *mb1, args, epi);
+  StreamArgs args{M, NP, n_tiles, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch, st.counters, status};
+  k_gemm_stream<BN, MT, Epi><<<grid, UM_THREADS, smem, stream>>>(*ma, *mb0, *mb1, args, epi);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
   return 0;
 }
 
-// True when the streaming kernel can take the problem: one row tile, K in whole 128-element chunks, and scratch and
-// counters large enough for its grid.
+// Row tiles the streaming kernel would use for M rows, or 0 when it cannot take the problem (more than 256 rows,
+// a tile too wide for two accumulators, or scratch / counters too small for its grid).
 template <typename Epi>
-bool stream_eligible(const UmmaState& st, int M, int NP, int K, int bn) {
-  if (!st.use_stream || M > UM_BM || K % ST_BK || st.scratch == nullptr) return false;
+int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn) {
+  if (!st.use_stream || M > 2 * UM_BM || st.scratch == nullptr) return 0;
+  const int mt = M > UM_BM ? 2 : 1;
+  if (mt * bn > 512 || (mt == 2 && !st.stream_two_tiles)) return 0;
   const int per_tile = Epi::kDual ? bn / 2 : bn;
   const int n_tiles = (NP + per_tile - 1) / per_tile;
-  return n_tiles <= st.n_counters && stream_scratch_bytes(stream_grid(st, n_tiles, M), bn) <= st.scratch_bytes;
+  if (n_tiles > st.n_counters || stream_scratch_bytes(stream_grid(st, n_tiles, M), bn, mt) > st.scratch_bytes) return 0;
+  return stream_shape(st, M, bn, mt, K).stages >= 2 ? mt : 0;
 }
 
 }  // namespace lsp

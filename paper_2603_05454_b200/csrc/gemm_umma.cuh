@@ -480,6 +480,11 @@ struct UmmaState {
   int skinny_min_stages = 3;       // ... provided each still gets this many pipeline stages
   int skinny_bn = 128;             // tile width of plain epilogues in that regime
   int use_stream = 1;              // M <= 128: use the persistent weight-streaming kernel (gemm_stream.cuh)
+  int stream_two_tiles = 1;        // ... also for 129..256 rows (two row tiles per CTA)
+  int stream_bn = 0;               // its tile width with one row tile (0 = automatic)
+  int stream_bn2 = 0;              // ... and with two row tiles
+  int stream_atoms = 0;            // K atoms per stage: 0 = two when stream_min_stages2 such stages fit, else 1 or 2 as given
+  int stream_min_stages2 = 3;
   int stream_grid_mode = 2;        // its grid: 0 = by row count, 1 = one CTA per SM (even shares), 2 = multiple of the tile count
   int stream_even_max_rows = 0;    // mode 0: even shares up to this many activation rows
   std::string err;
@@ -573,14 +578,14 @@ int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W
   return 0;
 }
 
-template <typename Epi> bool stream_eligible(const UmmaState& st, int M, int NP, int K, int bn);
-template <int BN, typename Epi>
+template <typename Epi> int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn);
+template <int BN, int MT, typename Epi>
 int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
-                  int n_rows_w, const Epi& epi, unsigned* status);
+                  int n_rows_w, const Epi& epi, unsigned* status, int box_rows);
 
 // Tile-width and split-K choice.
-//  * Problems with at most 128 activation rows go to the persistent weight-streaming kernel (gemm_stream.cuh) when it
-//    is eligible; the rules below cover the rest.
+//  * Problems with at most 256 activation rows go to the persistent weight-streaming kernel (gemm_stream.cuh) when it
+//    can take them; the rules below cover the rest.
 //  * Large problems (at least one CTA per SM without splitting) take the widest tile, one CTA per SM, deepest pipeline.
 //  * Single-row-tile problems (M <= 128) are bound by streaming the weights from HBM once.  Measured on B200, one
 //    CTA per SM that fetches 128 bytes per weight row per stage tops out near 3.7 TB/s however deep its pipeline is,
@@ -599,8 +604,11 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
     while (plan.a_rows < M) plan.a_rows *= 2;
   }
   if constexpr (Epi::kReduce) {
-    if (stream_eligible<Epi>(st, M, NP, K, UM_HEAD_BN))
-      return stream_launch<UM_HEAD_BN, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+    switch (stream_row_tiles<Epi>(st, M, NP, K, UM_HEAD_BN)) {
+      case 1: return stream_launch<UM_HEAD_BN, 1, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 0);
+      case 2: return stream_launch<UM_HEAD_BN, 2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 0);
+      default: break;
+    }
     if (mt == 1 && st.skinny_ctas_per_sm > 1) {
       const int stage = plan.a_rows * UM_BK * 2 + UM_HEAD_BN * UM_BK * 2;
       const int cap = (st.sm_smem / 2 - 1024) & ~1023;       // 2 x 256 accumulator columns fill the tensor memory
@@ -612,13 +620,32 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
     const int num_kb = K / UM_BK;
     int max_bn = 256;
     if constexpr (std::is_same<Epi, EpiQKVRope<bf16>>::value) max_bn = 2 * epi.half;
-    {
-      const int sbn = Epi::kDual ? max_bn : (max_bn < 128 ? max_bn : 128);
-      if (stream_eligible<Epi>(st, M, NP, K, sbn)) {
+    if (M <= 2 * UM_BM) {
+      // Tile width, from measurements on the LLaDA layer shapes at 2..256 rows: dual epilogues take 256 columns (128
+      // pairs); plain ones take 128, which needs no K split with 96 tiles, except that a wide GEMM with at most 32
+      // rows takes 256 (its partial tiles are small, and half as many MMA instructions are issued).  The rotary
+      // epilogue's half tiles are fetched head by head.
+      int sbn = Epi::kDual ? 256 : ((M <= 32 && cols >= 8192) ? 256 : 128), box_rows = 0;
+      if constexpr (std::is_same<Epi, EpiQKVRope<bf16>>::value) {
+        box_rows = epi.half;
+        sbn = (M <= 32) ? 256 : 128;
+      }
+      if (M <= UM_BM && st.stream_bn > 0) sbn = st.stream_bn;
+      if (M > UM_BM && st.stream_bn2 > 0) sbn = st.stream_bn2;
+      if (box_rows > sbn / 2) sbn = 2 * box_rows;
+      const int smt = stream_row_tiles<Epi>(st, M, NP, K, sbn);
+      if (smt == 1) {
         switch (sbn) {
-          case 256: return stream_launch<256, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
-          case 128: return stream_launch<128, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
-          case 64: return stream_launch<64, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status);
+          case 256: return stream_launch<256, 1, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
+          case 128: return stream_launch<128, 1, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
+          case 64: return stream_launch<64, 1, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
+          default: break;
+        }
+      } else if (smt == 2) {
+        switch (sbn) {
+          case 256: return stream_launch<256, 2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
+          case 128: return stream_launch<128, 2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
+          case 64: return stream_launch<64, 2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
           default: break;
         }
       }

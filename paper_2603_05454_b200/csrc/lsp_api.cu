@@ -154,7 +154,7 @@ struct Layout {
       gemm_scratch, gemm_counters, stage, total;
 };
 
-constexpr size_t kGemmScratchBytes = 64u << 20;   // split-K partial tiles
+constexpr size_t kGemmScratchBytes = 80u << 20;   // split-K partial tiles (the streaming GEMM needs 74 MiB at its widest)
 constexpr int kGemmCounters = 4096;               // split-K arrival counters
 
 int head_tiles_max(const lsp_model_cfg* m) { return (m->vocab + 63) / 64; }
@@ -619,6 +619,11 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   else if (key == 16) c->umma.use_stream = value;
   else if (key == 17) c->umma.stream_grid_mode = value;
   else if (key == 18) c->umma.stream_even_max_rows = value;
+  else if (key == 19) c->umma.stream_two_tiles = value;
+  else if (key == 20) c->umma.stream_bn2 = (value == 256 || value == 128 || value == 64) ? value : 0;
+  else if (key == 23) c->umma.stream_bn = (value == 256 || value == 128 || value == 64) ? value : 0;
+  else if (key == 21) c->umma.stream_atoms = value;
+  else if (key == 22) c->umma.stream_min_stages2 = value < 2 ? 2 : value;
   else if (key == 13) c->umma.skinny_ctas_per_sm = value < 1 ? 1 : value;
   else if (key == 14) c->umma.skinny_min_stages = value < 1 ? 1 : value;
   else if (key == 15) c->umma.skinny_bn = (value == 64 || value == 32) ? value : 128;

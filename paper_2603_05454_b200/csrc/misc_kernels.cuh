@@ -34,30 +34,98 @@ __global__ void k_assemble_embed(StepDesc sd, int batch, const int32_t* __restri
 
 // ---------------------------------------------------------------------------------------------
 // RMSNorm: out[r] = x[src[r]] / sqrt(mean(x^2) + eps) * g, fp32 arithmetic, one block per output row.
+// The row is read once with 128-bit loads and kept in registers between the reduction and the scaling
+// (up to RN_VPT vectors per thread; longer rows fall back to a second read).
 // ---------------------------------------------------------------------------------------------
+constexpr int RN_THREADS = 256;
+constexpr int RN_VPT = 4;      // 16-byte vectors per thread held in registers
+
+template <typename T> struct Vec16 { static constexpr int N = 16 / (int)sizeof(T); };
+
+__device__ __forceinline__ void vec_to_f(const uint4& u, float (&v)[4]) {
+  v[0] = __uint_as_float(u.x); v[1] = __uint_as_float(u.y); v[2] = __uint_as_float(u.z); v[3] = __uint_as_float(u.w);
+}
+__device__ __forceinline__ void vec_to_f(const uint4& u, float (&v)[8]) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { v[2 * i] = __low2float(p[i]); v[2 * i + 1] = __high2float(p[i]); }
+}
+__device__ __forceinline__ uint4 f_to_vec(const float (&v)[4]) {
+  return make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+}
+__device__ __forceinline__ uint4 f_to_vec(const float (&v)[8]) {
+  uint4 r;
+  __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+  __nv_bfloat162 c = __floats2bfloat162_rn(v[4], v[5]), d = __floats2bfloat162_rn(v[6], v[7]);
+  r.x = *reinterpret_cast<uint32_t*>(&a); r.y = *reinterpret_cast<uint32_t*>(&b);
+  r.z = *reinterpret_cast<uint32_t*>(&c); r.w = *reinterpret_cast<uint32_t*>(&d);
+  return r;
+}
+
 template <typename T>
-__global__ void k_rmsnorm(const T* __restrict__ x, const T* __restrict__ g, T* __restrict__ out,
-                          const int* __restrict__ src_rows, int d, float eps) {
-  __shared__ float red[32];
+__global__ void __launch_bounds__(RN_THREADS) k_rmsnorm(const T* __restrict__ x, const T* __restrict__ g, T* __restrict__ out,
+                                                       const int* __restrict__ src_rows, int d, float eps) {
+  constexpr int E = Vec16<T>::N;                 // elements per 16-byte vector
+  __shared__ float red[RN_THREADS / 32];
   const int r = blockIdx.x;
-  const T* xr = x + (size_t)(src_rows ? src_rows[r] : r) * d;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)(src_rows ? src_rows[r] : r) * d);
+  const uint4* gr = reinterpret_cast<const uint4*>(g);
+  uint4* o = reinterpret_cast<uint4*>(out + (size_t)r * d);
+  const int nv = d / E;                          // d is a multiple of 64
+  const bool in_regs = nv <= RN_VPT * RN_THREADS;
+  uint4 keep[RN_VPT];
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    const float v = to_f(xr[i]);
-    ss += v * v;
+  if (in_regs) {
+#pragma unroll
+    for (int j = 0; j < RN_VPT; ++j) {
+      const int i = threadIdx.x + j * RN_THREADS;
+      keep[j] = (i < nv) ? xr[i] : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int j = 0; j < RN_VPT; ++j) {
+      float v[E];
+      vec_to_f(keep[j], v);
+#pragma unroll
+      for (int e = 0; e < E; ++e) ss += v[e] * v[e];
+    }
+  } else {
+    for (int i = threadIdx.x; i < nv; i += RN_THREADS) {
+      float v[E];
+      vec_to_f(xr[i], v);
+#pragma unroll
+      for (int e = 0; e < E; ++e) ss += v[e] * v[e];
+    }
   }
   ss = warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
-  if (threadIdx.x < 32) {
-    float v = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
-    v = warp_sum(v);
-    if (threadIdx.x == 0) red[0] = v;
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < RN_THREADS / 32; ++w) tot += red[w];      // same order in every thread
+  const float inv = rsqrtf(tot / (float)d + eps);
+  if (in_regs) {
+#pragma unroll
+    for (int j = 0; j < RN_VPT; ++j) {
+      const int i = threadIdx.x + j * RN_THREADS;
+      if (i < nv) {
+        float v[E], gv[E];
+        vec_to_f(keep[j], v);
+        vec_to_f(__ldg(gr + i), gv);
+#pragma unroll
+        for (int e = 0; e < E; ++e) v[e] = v[e] * inv * gv[e];
+        o[i] = f_to_vec(v);
+      }
+    }
+  } else {
+    for (int i = threadIdx.x; i < nv; i += RN_THREADS) {
+      float v[E], gv[E];
+      vec_to_f(xr[i], v);
+      vec_to_f(__ldg(gr + i), gv);
+#pragma unroll
+      for (int e = 0; e < E; ++e) v[e] = v[e] * inv * gv[e];
+      o[i] = f_to_vec(v);
+    }
   }
-  __syncthreads();
-  const float inv = rsqrtf(red[0] / (float)d + eps);
-  T* o = out + (size_t)r * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) o[i] = from_f<T>(to_f(xr[i]) * inv * to_f(g[i]));
 }
 
 // ---------------------------------------------------------------------------------------------

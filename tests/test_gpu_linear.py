@@ -57,9 +57,10 @@ def test_linear_bf16(impl, shape):
 
 @pytest.mark.parametrize("grid_mode", [1, 2])
 @pytest.mark.parametrize("shape", [(1, 256, 128), (5, 384, 256), (64, 1152, 512), (128, 4096, 4096), (100, 12288, 4096),
-                                   (17, 4096, 12288)])
+                                   (17, 4096, 12288), (129, 384, 256), (200, 4096, 4096), (256, 12288, 4096),
+                                   (190, 1152, 576)])
 def test_linear_bf16_weight_streaming_kernel(grid_mode, shape):
-    """M <= 128 and K in whole 128-element chunks take the persistent streaming kernel: tiles split between CTAs
+    """M <= 256 takes the persistent streaming kernel (one or two row tiles per CTA): tiles split between CTAs
     (partials in scratch, summed by the last arriver) with both ways of dealing out the work."""
     M, N, K = shape
     tdt = torch.bfloat16
