@@ -211,6 +211,25 @@ int lsp_last_timing(lsp_ctx* ctx, float* ms);
 int lsp_get_counters(lsp_ctx* ctx, double* out);
 int lsp_reset_counters(lsp_ctx* ctx);
 
+/* (No counterpart in the paper: a convenience for callers that cannot allocate.)
+ * out[M, N] = A[M, K] W[N, K]^T in bfloat16 with fp32 accumulation, without a context and without any allocation:
+ * the split-K partial tiles and tile counters that lsp_op_linear keeps in the caller's workspace live here in a
+ * static array inside the library's device image (8 MiB + 16 KiB; every GPU that loads the library holds it until
+ * the process exits).  It is meant for code that runs where cudaMalloc is off limits, such as a plug-in called inside
+ * another framework's memory pool or from a real-time loop, and therefore cannot create the workspace lsp_init() needs.
+ *   A, W, out  device pointers, 16-byte aligned, row-major, bfloat16; out is written completely.
+ *   limits     1 <= M <= 128; N a multiple of 16, at most 524288; K a multiple of 64.  Anything else returns
+ *              LSP_ERR_SHAPE (NULL or misaligned pointers: LSP_ERR_ARG) and writes a message into err.
+ *   cuda_stream  a cudaStream_t (NULL = default stream); the call only enqueues work and returns.
+ *   err, err_len  optional host buffer that receives a message when the call fails.
+ * The first call on a device looks up the array's device address and sets a kernel attribute, once, with that
+ * device current; make that first call outside any stream capture.  Every call uses the same array: it clears the
+ * counters itself (so a call that was aborted leaves nothing behind), but two calls whose kernels overlap on the GPU,
+ * from different streams or threads, race on it and give wrong results; calls on one stream are safe.  The call
+ * itself performs no cudaMalloc/cudaFree and uses no allocating library routine. */
+int lsp_linear_static(const void* A, const void* W, void* out, int M, int N, int K, void* cuda_stream, char* err,
+                      size_t err_len);
+
 const char* lsp_last_error(const lsp_ctx* ctx);
 int lsp_destroy(lsp_ctx* ctx);
 

@@ -4,7 +4,7 @@ The Python layer only marshals arguments; every step of the path runs in the lib
 The binding is imported on first use and fails loudly when the compiled library is missing
 (`python -m paper_2603_05454_b200.build` builds it); there is no CPU or PyTorch fallback.
 """
-_NAMES = ("LSPDecoder", "SchedCfg", "lib", "LSPError", "FLAG_SNAPPED", "FLAG_FALLBACK", "FLAG_RANGE_UNACHIEVABLE",
+_NAMES = ("LSPDecoder", "SchedCfg", "lib", "LSPError", "linear_static", "FLAG_SNAPPED", "FLAG_FALLBACK", "FLAG_RANGE_UNACHIEVABLE",
           "FLAG_RUN_TO_END", "FLAG_NEAR_THRESHOLD", "FLAG_NEAR_TIE")
 __all__ = list(_NAMES)
 

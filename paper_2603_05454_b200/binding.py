@@ -18,7 +18,7 @@ FLAG_RUN_TO_END, FLAG_NEAR_THRESHOLD, FLAG_NEAR_TIE = 8, 16, 32
 EXPORTS = ["lsp_workspace_bytes", "lsp_kv_cache_bytes", "lsp_init", "lsp_set_sched", "lsp_set_option",
            "lsp_begin", "lsp_denoise_step", "lsp_commit", "lsp_generate", "lsp_generate_host", "lsp_active", "lsp_score_rows",
            "lsp_get_scores", "lsp_head_scan", "lsp_scan", "lsp_op_linear", "lsp_last_timing", "lsp_get_counters", "lsp_reset_counters",
-           "lsp_last_error", "lsp_destroy"]
+           "lsp_linear_static", "lsp_last_error", "lsp_destroy"]
 
 
 class LSPError(RuntimeError):
@@ -76,6 +76,8 @@ def _load():
     l.lsp_last_timing.argtypes = [C.c_void_p, C.c_void_p]
     l.lsp_get_counters.argtypes = [C.c_void_p, C.c_void_p]
     l.lsp_reset_counters.argtypes = [C.c_void_p]
+    l.lsp_linear_static.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_char_p,
+                                    C.c_size_t]
     l.lsp_last_error.restype = C.c_char_p
     l.lsp_last_error.argtypes = [C.c_void_p]
     l.lsp_destroy.argtypes = [C.c_void_p]
@@ -292,6 +294,20 @@ class LSPDecoder:
     def kv_view(self):
         s = self.shape
         return self.kv_cache.view(self.tdtype).view(s.n_layers, 2, self.max_batch, self.max_len, s.n_kv_heads, s.head_dim)
+
+
+def linear_static(A: torch.Tensor, W: torch.Tensor, out: torch.Tensor, stream=None):
+    """out = A W^T through lsp_linear_static: no context, no workspace; the library's static scratch is used.
+    A [M, K], W [N, K], out [M, N]: contiguous bfloat16 CUDA tensors on the current device."""
+    M, K = A.shape
+    N = W.shape[0]
+    sptr = stream.cuda_stream if stream is not None else torch.cuda.current_stream(A.device).cuda_stream
+    buf = C.create_string_buffer(256)
+    with torch.cuda.device(A.device):
+        rc = lib.lsp_linear_static(A.data_ptr(), W.data_ptr(), out.data_ptr(), M, N, K, sptr, buf, len(buf))
+    if rc != 0:
+        raise LSPError(rc, buf.value.decode())
+    return out
 
 
 def _rec(r: StepRec):

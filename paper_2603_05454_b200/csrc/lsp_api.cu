@@ -5,6 +5,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <type_traits>
 #include <string>
 #include <vector>
@@ -855,6 +856,133 @@ int lsp_reset_counters(lsp_ctx* c) {
   seg_collect(c);
   memset(c->counters, 0, sizeof c->counters);
   memset(c->timing_ms, 0, sizeof c->timing_ms);
+  return LSP_OK;
+}
+
+// ---- lsp_linear_static: the streaming GEMM with its scratch in a static device array ----------------------------
+namespace {
+
+constexpr int kStaticMaxCtas = 64;        // CTAs the static variant launches at most
+constexpr int kStaticBN = 128;            // its tile width
+constexpr int kStaticMaxTiles = 4096;     // tile counters
+constexpr size_t kStaticPartialBytes = (size_t)kStaticMaxCtas * 2 * UM_BM * kStaticBN * sizeof(float);   // 8 MiB
+constexpr size_t kStaticScratchBytes = kStaticPartialBytes + (size_t)kStaticMaxTiles * sizeof(unsigned) + 256;
+
+// Partial tiles, then the tile counters, then the status word.  One copy per GPU that loads the library, held until
+// the process exits.  In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kStaticMaxDevices = 64;
+struct StaticDev {
+  std::once_flag once;
+  cudaError_t setup_rc = cudaErrorUnknown;
+  unsigned char* scratch = nullptr;      // device address of g_static_scratch on this device
+  PFN_encodeTiled encode = nullptr;
+  int max_smem = 0, n_sm = 0;
+};
+StaticDev g_static_dev[kStaticMaxDevices];
+
+void static_msg(char* err, size_t err_len, const char* fmt, ...) {
+  if (!err || err_len == 0) return;
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(err, err_len, fmt, ap);
+  va_end(ap);
+}
+
+bool static_map(PFN_encodeTiled encode, CUtensorMap* m, const void* base, int rows, int K, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)UM_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int lsp_linear_static(const void* A, const void* W, void* out, int M, int N, int K, void* cuda_stream, char* err,
+                      size_t err_len) {
+  if (err && err_len) err[0] = 0;
+  if (!A || !W || !out) { static_msg(err, err_len, "lsp_linear_static: NULL pointer"); return LSP_ERR_ARG; }
+  if (M < 1 || M > UM_BM || N < 16 || N % 16 || K < 64 || K % 64 || (N + kStaticBN - 1) / kStaticBN > kStaticMaxTiles) {
+    static_msg(err, err_len,
+               "lsp_linear_static: M = %d, N = %d, K = %d outside the static scratch's limits (1 <= M <= %d, N a multiple "
+               "of 16 up to %d, K a multiple of 64)", M, N, K, UM_BM, kStaticMaxTiles * kStaticBN);
+    return LSP_ERR_SHAPE;
+  }
+  if (((uintptr_t)A | (uintptr_t)W | (uintptr_t)out) & 15) {
+    static_msg(err, err_len, "lsp_linear_static: pointers must be 16-byte aligned");
+    return LSP_ERR_ARG;
+  }
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) {
+    static_msg(err, err_len, "lsp_linear_static: no usable current device (%s)", cudaGetErrorString(e));
+    return LSP_ERR_CUDA;
+  }
+  StaticDev& sd = g_static_dev[dev];
+  // First call on this device (with that device current): resolve the device address of the static array.
+  std::call_once(sd.once, [&sd, dev]() {
+    void* p = nullptr;
+    cudaError_t rc = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (rc == cudaSuccess) {
+      sd.scratch = (unsigned char*)p;
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult q;
+      rc = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+      if (rc == cudaSuccess && (fn == nullptr || q != cudaDriverEntryPointSuccess)) rc = cudaErrorNotSupported;
+      sd.encode = (PFN_encodeTiled)fn;
+    }
+    if (rc == cudaSuccess) rc = cudaDeviceGetAttribute(&sd.max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (rc == cudaSuccess) rc = cudaDeviceGetAttribute(&sd.n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (rc == cudaSuccess)
+      rc = cudaFuncSetAttribute(k_gemm_stream<kStaticBN, 1, EpiStore<bf16>>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                sd.max_smem);
+    sd.setup_rc = rc;
+  });
+  if (sd.setup_rc != cudaSuccess) {
+    static_msg(err, err_len, "lsp_linear_static: set-up on device %d failed (%s)", dev, cudaGetErrorString(sd.setup_rc));
+    return LSP_ERR_CUDA;
+  }
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  // stage shape: as many two-atom stages as fit, else one-atom stages
+  const int a_rows = (M + 7) / 8 * 8;
+  const int aux = 1024 + UM_BM * 128 + 8 * (2 * ST_MAX_STAGES + 4) + 16;
+  const int atom = a_rows * 128 + kStaticBN * 128;
+  const int atoms = (K % 128 == 0 && (sd.max_smem - aux) / (2 * atom) >= 3) ? 2 : 1;
+  int stages = (sd.max_smem - aux) / (atoms * atom);
+  if (stages > ST_MAX_STAGES) stages = ST_MAX_STAGES;
+  const size_t smem = (size_t)stages * atoms * atom + aux;
+  CUtensorMap ma, mb;
+  if (stages < 2 || !static_map(sd.encode, &ma, A, M, K, a_rows) || !static_map(sd.encode, &mb, W, N, K, kStaticBN / 2)) {
+    static_msg(err, err_len, "lsp_linear_static: could not describe the operands to the copy engine");
+    return LSP_ERR_CUDA;
+  }
+  const int n_tiles = (N + kStaticBN - 1) / kStaticBN;
+  const int kc = K / (atoms * UM_BK);
+  const long U = (long)n_tiles * kc;
+  const int max_ctas = sd.n_sm < kStaticMaxCtas ? sd.n_sm : kStaticMaxCtas;
+  int grid = n_tiles <= max_ctas ? n_tiles * (max_ctas / n_tiles) : max_ctas;
+  if (grid > U) grid = (int)U;
+  float* partials = (float*)sd.scratch;
+  unsigned* counters = (unsigned*)(sd.scratch + kStaticPartialBytes);
+  unsigned* status = counters + kStaticMaxTiles;
+  // the array keeps whatever the last call left: the counters (and the status word) must start at zero
+  e = cudaMemsetAsync(counters, 0, (size_t)kStaticMaxTiles * sizeof(unsigned) + 16, stream);
+  if (e != cudaSuccess) {
+    static_msg(err, err_len, "lsp_linear_static: clearing the counters failed (%s)", cudaGetErrorString(e));
+    return LSP_ERR_CUDA;
+  }
+  StreamArgs args{M, N, n_tiles, kc, a_rows, atoms, kStaticBN / 2, stages, partials, counters, status};
+  EpiStore<bf16> epi{(bf16*)out, N};
+  k_gemm_stream<kStaticBN, 1, EpiStore<bf16>><<<grid, UM_THREADS, smem, stream>>>(ma, mb, mb, args, epi);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    static_msg(err, err_len, "lsp_linear_static: launch failed (%s)", cudaGetErrorString(e));
+    return LSP_ERR_CUDA;
+  }
   return LSP_OK;
 }
 
