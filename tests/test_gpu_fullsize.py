@@ -1,0 +1,83 @@
+"""Parity at the benchmark configurations' full widths, on outputs the oracle can afford to compute.
+
+ * cfg2 (fused LM head + confidence + scan, hidden [8 x 1024, 4096], vocabulary 126464): the oracle computes full
+   fp64 logits only for sampled rows and for the left end of every sequence up to one row past the first position that
+   fails the threshold, which is all the scan's result depends on.
+ * LLaDA-8B- and Dream-7B-shaped layers (full d_model, heads, FFN width; one layer, small vocabulary): teacher-forced
+   decode steps whose row counts cover the tiled GEMM (more than 256 rows) and both shapes of the streaming GEMM.
+"""
+import numpy as np
+import pytest
+import torch
+
+import lsp_synth as S
+from oracle import scan as oscan
+from oracle.scores import scores_from_logits
+from gpu_util import DEV, tol_for, tol_logit
+from test_gpu_decode import _teacher_forced
+
+pytestmark = pytest.mark.gpu
+NEAR = oscan.FLAG_NEAR_THRESHOLD | oscan.FLAG_NEAR_TIE
+
+
+def test_cfg2_full_size_head_and_scan_on_sampled_rows_and_run_prefixes():
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+    d, V, B, L, tau, scale = 4096, 126464, 8, 1024, 0.9, 6.0
+    sh = S.ModelShape(1, d, 32, 32, 128, 64, V, dtype="bf16", head_scale=scale)
+    z = lambda *s: torch.zeros(*s, dtype=torch.bfloat16, device=DEV)
+    w = dict(embed=z(8, d), w_head=S.normal((V, d), 0, S.TID_HEAD, 0.02 * scale, torch.bfloat16, DEV),
+             final_norm=torch.ones(d, dtype=torch.bfloat16, device=DEV),
+             layers=[dict(attn_norm=z(d), w_qkv=z(3 * d, d), w_o=z(d, d), ffn_norm=z(d), w_gate=z(64, d), w_up=z(64, d),
+                          w_down=z(d, 64))])
+    hidden = S.normal((B * L, d), 0, 77, 1.0, torch.bfloat16, DEV)
+    w64 = w["w_head"].float().cpu().numpy().astype(np.float64)
+    h_cpu = hidden.float().cpu().numpy().astype(np.float64)
+    tol = tol_for("bf16")
+    # identical inputs on both sides: only the accumulation order differs
+    tol_z = tol_logit("fp32", 0.02 * scale * np.sqrt(d))
+    sched = SchedCfg(tau=tau, delim_bitmap=S.delimiter_bitmap(V, 1, 32).to(DEV), flag_tol=tol, tie_tol=tol_z)
+    dec = LSPDecoder(sh, w, sched, B, L, device=DEV)
+    off = np.arange(B + 1, dtype=np.int32) * L
+    out = dec.head_scan(hidden, off)
+    y, p, m = dec.scores()
+    dec.close()
+
+    def oracle_rows(rows):
+        return scores_from_logits(h_cpu[rows] @ w64.T, sh.mask_id)
+
+    # (a) sampled rows anywhere (several row tiles, both ends)
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, 129, B * L - 1], (np.arange(40) * 204 + 7) % (B * L)]))
+    yo, po, mo = oracle_rows(rows)
+    assert np.abs(p[rows] - po).max() <= 1e-4
+    assert np.abs(m[rows] - mo).max() <= tol_z
+    assert all(mo[i] <= tol_z for i in np.nonzero(y[rows] != yo)[0])
+    # (b) every sequence's run: oracle scores from the left until one row past the first failure
+    for b in range(B):
+        n = 32
+        while True:
+            yo, po, mo = oracle_rows(np.arange(off[b], off[b] + n))
+            if (po < tau).any() or n >= L:
+                break
+            n = min(L, 2 * n)
+        first_fail = int(np.argmax(po < tau)) if (po < tau).any() else n
+        keep = min(n, first_fail + 2)
+        r = oscan.lsp_scan(po[:keep], yo[:keep], lambda t: 1 <= t <= 32, tau=float(np.float32(tau)), W=16,
+                           flag_tol=float(np.float32(tol)), tie_tol=float(np.float32(tol_z)), margin=mo[:keep])
+        if r["flags"] & NEAR:
+            continue
+        # a truncated sequence can only differ from the full one in the run-to-end rule, which needs L' = keep
+        assert r["L_run"] < keep
+        assert (out["L_run"][b], out["L_commit"][b]) == (r["L_run"], r["L_commit"]), (b, out, r)
+
+
+@pytest.mark.parametrize("name", ["llada", "dream"])
+def test_full_width_layer_teacher_forced_steps(name):
+    from paper_2603_05454_b200 import SchedCfg
+    if name == "llada":
+        sh = S.ModelShape(1, 4096, 32, 32, 128, 12288, 8192, dtype="bf16", head_scale=4.0)
+    else:
+        sh = S.ModelShape(1, 3584, 28, 4, 128, 18944, 8192, dtype="bf16", head_scale=4.0, rope_theta=1e6)
+    # pass 0 has 300 rows (tiled GEMM, three row tiles), pass 1 about 250 (streaming GEMM, two row tiles); the
+    # fixed-k policy then walks the row count down through the one-row-tile regime
+    _teacher_forced(sh, 21, 50, 250, SchedCfg(tau=0.9), (1, 64), max_steps=2)
+    _teacher_forced(sh, 22, 8, 150, SchedCfg(mode=2, fixed_k=60), (1, 64), max_steps=3)
