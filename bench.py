@@ -435,7 +435,7 @@ def main():
             "tokens_per_pass": r["l_commit_mean"],
             "roofline": {"bound": "hbm", "achieved": gemm.get("gbs"), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": gemm.get("hbm_frac"), "traffic": gemm.get("traffic"),
-                         "kernel": "k_gemm_umma (layer projections and FFN; weight-streaming regime, rows <= 512)",
+                         "kernel": "k_gemm_stream (layer projections and FFN; all but the first pass have at most 257 rows: weight-streaming regime)",
                          "peak_kind": "of " + peak_kind,
                          "timed": "per-launch CUDA events, second pass over the same K decodes"},
             "classes": r["classes"],

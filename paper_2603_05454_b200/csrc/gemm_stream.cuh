@@ -1,4 +1,5 @@
-// Weight-streaming bf16 GEMM for at most 256 activation rows (the shrinking suffix of late decode steps), tcgen05.
+// Persistent bf16 GEMM on tcgen05, built for the weight-streaming regime (at most 256 activation rows: the shrinking
+// suffix of late decode steps) and also used, with whole tiles per CTA, for larger problems.
 //
 //   acc[m, c] = sum_k A[m, k] * Wt[c, k]        same operands, tiles and fused epilogues as gemm_umma.cuh
 //
@@ -34,6 +35,9 @@ struct StreamArgs {
   int M;            // activation rows (<= 128 MT)
   int n_pairs;      // dual: pair indices; plain: output columns
   int n_tiles;      // column tiles
+  int row_groups;   // groups of 128 MT activation rows (1 when M <= 128 MT); a tile is (column tile, row group), row
+                    // group fastest, so a CTA meets the same weight tile again while it is still in L2
+  int whole_tiles;  // 1: shares are whole tiles (no tile is split between CTAs)
   int kc;           // K chunks (one per stage) per tile
   int a_rows;       // activation box rows (M rounded up to a multiple of 8)
   int atoms;        // 64-element K atoms per stage (1 or 2)
@@ -108,21 +112,31 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   const uint32_t tmem_base = *tmem_slot;
 
   const int G = gridDim.x, g = blockIdx.x;
-  const long U = (long)args.n_tiles * args.kc;
-  const long u0 = st_first_unit(U, G, g), u1 = st_first_unit(U, G, g + 1);
+  const int RG = args.row_groups;
+  const long T = (long)args.n_tiles * RG;
+  const long U = T * args.kc;
+  // Split shares: CTA g owns the contiguous units [U g / G, U (g + 1) / G).  Whole-tile shares: CTA g owns tiles
+  // g, g + G, g + 2 G, ... (units are then counted within its own tiles), so that the CTAs running at any moment work
+  // on neighbouring tiles: the same few weight tiles for every row group, which keeps the working set inside L2.
+  const long u0 = args.whole_tiles ? 0 : st_first_unit(U, G, g);
+  const long u1 = args.whole_tiles ? ((T - g + G - 1) / G) * args.kc : st_first_unit(U, G, g + 1);
 
   if (warp == 0) {
     // ---------------- TMA producer: one uninterrupted stream over this CTA's units ----------------
     if (lane == 0) {
       long issued = 0;
-      for (long u = u0; u < u1; ++u) {
-        const int it = (int)(u - u0), s = it % S;
-        const uint32_t ph = (uint32_t)(it / S) & 1u;
+      // position in the unit space, advanced without divisions (this loop has to keep ahead of the tensor pipe)
+      int vt = (int)(u0 / args.kc), c = (int)(u0 % args.kc);
+      int tlin = args.whole_tiles ? g + vt * G : vt;
+      int tile = tlin / RG, rg = tlin % RG;
+      int s = 0;
+      uint32_t ph = 0;
+      const int n_units = (int)(u1 - u0);
+      for (int it = 0; it < n_units; ++it) {
         if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
           if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 11u; }
           break;
         }
-        const int tile = (int)(u / args.kc), c = (int)(u % args.kc);
         mbar_expect_tx(full_bar(s), STAGE_BYTES);
         const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
         const uint32_t sb = sa + AT * A_ATOM;
@@ -136,8 +150,16 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
           for (int j = 0; j < AT; ++j)
             tma_load_2d(sb + j * B_ATOM + B_HALF_ATOM + b * 128, &map_b1, k0 + 64 * j, row_b1, full_bar(s));
         }
-        for (int j = 0; j < AT; ++j) tma_load_2d(sa + j * A_ATOM, &map_a, k0 + 64 * j, 0, full_bar(s));
+        for (int j = 0; j < AT; ++j) tma_load_2d(sa + j * A_ATOM, &map_a, k0 + 64 * j, rg * ROWS, full_bar(s));
         ++issued;
+        if (++s == S) { s = 0; ph ^= 1u; }
+        if (++c == args.kc) {
+          c = 0;
+          ++vt;
+          tlin = args.whole_tiles ? g + vt * G : vt;
+          tile = tlin / RG;
+          rg = tlin % RG;
+        }
       }
       // do not leave while copies may still be landing in this CTA's shared memory
       const long first = issued > S ? issued - S : 0;
@@ -152,9 +174,11 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
       constexpr uint32_t idesc = make_idesc(BN);
       int seg = 0;
       bool ok = true;
+      int s = 0;
+      uint32_t ph = 0;
       for (long u = u0; u < u1 && ok;) {
-        const int tile = (int)(u / args.kc);
-        const long seg_end = min(u1, (long)(tile + 1) * args.kc);
+        const int vt = (int)(u / args.kc);
+        const long seg_end = min(u1, (long)(vt + 1) * args.kc);
         const int buf = seg % NBUF, use = seg / NBUF;
         // wait until the epilogue has drained this accumulator set (its previous use was segment seg - NBUF)
         if (use >= 1 && !mbar_wait(acce_bar(buf), (uint32_t)(use - 1) & 1u, abort_flag)) {
@@ -166,8 +190,6 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
         bool first = true;
         for (; u < seg_end; ++u) {
-          const int it = (int)(u - u0), s = it % S;
-          const uint32_t ph = (uint32_t)(it / S) & 1u;
           if (!mbar_wait(full_bar(s), ph, abort_flag)) {
             if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 13u; }
             ok = false;
@@ -189,6 +211,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             }
           }
           tc_commit(empty_bar(s));
+          if (++s == S) { s = 0; ph ^= 1u; }
         }
         if (ok) tc_commit(accf_bar(buf));
         ++seg;
@@ -202,8 +225,10 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     int seg = 0;
     bool ok = true;
     for (long u = u0; u < u1 && ok; ++seg) {
-      const int tile = (int)(u / args.kc);
-      const long tile_u0 = (long)tile * args.kc;
+      const int vt = (int)(u / args.kc);
+      const int tlin = args.whole_tiles ? g + vt * G : vt;
+      const int tile = tlin / RG, row0 = (tlin % RG) * ROWS;      // column tile, first activation row
+      const long tile_u0 = (long)vt * args.kc;
       const long seg_end = min(u1, tile_u0 + args.kc);
       const bool whole = (u == tile_u0) && (seg_end == tile_u0 + args.kc);
       const int buf = seg % NBUF, use = seg / NBUF;
@@ -219,7 +244,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         // the accumulator is complete in tensor memory: each thread owns one row of every row tile
 #pragma unroll 1
         for (int mt = 0; mt < MT; ++mt) {
-          const int m = mt * UM_BM + r_in;
+          const int m = row0 + mt * UM_BM + r_in;
           Top2 red = top2_empty();
 #pragma unroll 1
           for (int c = 0; c < CH; c += 16) {
@@ -374,11 +399,12 @@ inline int stream_grid(const UmmaState& st, int n_tiles, int M) {
   return M <= st.stream_even_max_rows ? st.n_sm : aligned;
 }
 
-// Stage shape for M rows and tile width bn: two K atoms per stage when at least three such stages fit.
+// Stage shape for an activation box of a_rows rows and tile width bn: two K atoms per stage when at least
+// stream_min_stages2 such stages fit.
 struct StreamShape { int a_rows, atoms, stages, stage_bytes, aux; };
-inline StreamShape stream_shape(const UmmaState& st, int M, int bn, int mt, int K) {
+inline StreamShape stream_shape(const UmmaState& st, int a_rows, int bn, int mt, int K) {
   StreamShape sh;
-  sh.a_rows = (M + 7) / 8 * 8;
+  sh.a_rows = a_rows;
   sh.aux = 1024 + UM_BM * mt * 128 + 8 * (2 * ST_MAX_STAGES + 4) + 16;
   const int atom = sh.a_rows * 128 + bn * 128;
   sh.atoms = (K % 128 == 0 && (st.max_smem - sh.aux) / (2 * atom) >= st.stream_min_stages2) ? 2 : 1;
@@ -389,11 +415,13 @@ inline StreamShape stream_shape(const UmmaState& st, int M, int bn, int mt, int 
   if (sh.stages > st.max_stages) sh.stages = st.max_stages;
   return sh;
 }
+// Activation box rows: all rows (rounded up to 8) when they fit one group of 128 mt rows, else a full group.
+inline int stream_a_rows(int M, int mt) { return M <= UM_BM * mt ? (M + 7) / 8 * 8 : UM_BM * mt; }
 
 template <int BN, int MT, typename Epi>
 int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
                   int n_rows_w, const Epi& epi, unsigned* status, int box_rows) {
-  const StreamShape sh = stream_shape(st, M, BN, MT, K);
+  const StreamShape sh = stream_shape(st, stream_a_rows(M, MT), BN, MT, K);
   if (sh.stages < 2) { st.err = "not enough shared memory for the streaming GEMM"; return -2; }
   const size_t smem = (size_t)sh.stages * sh.stage_bytes + sh.aux;
   static bool attr_set = false;   // per instantiation
@@ -403,35 +431,56 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
     attr_set = true;
   }
   if (st.cache.size() > 4096) st.cache.clear();
-  const CUtensorMap* ma = umma_map(st, A, M, K, sh.a_rows);
   if (box_rows <= 0 || box_rows > BN / 2 || (BN / 2) % box_rows || box_rows % 8) box_rows = BN / 2;
+  const CUtensorMap* ma = umma_map(st, A, M, K, sh.a_rows);
   const CUtensorMap* mb0 = umma_map(st, W0, n_rows_w, K, box_rows);
   const CUtensorMap* mb1 = umma_map(st, W1, n_rows_w, K, box_rows);
   if (!ma || !mb0 || !mb1) return -4;
   const int per_tile = Epi::kDual ? BN / 2 : BN;
   const int n_tiles = (NP + per_tile - 1) / per_tile;
   const int kc = K / (sh.atoms * UM_BK);
-  long U = (long)n_tiles * kc;
-  int grid = stream_grid(st, n_tiles, M);
-  if (grid > U) grid = (int)U;
-  StreamArgs args{M, NP, n_tiles, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch, st.counters, status};
+  const int row_groups = (M + UM_BM * MT - 1) / (UM_BM * MT);
+  // several row groups: whole tiles per CTA (the problem is large enough); one row group: K slices as stream_grid says
+  const int whole = row_groups > 1 ? 1 : 0;
+  const long T = (long)n_tiles * row_groups;
+  int grid = whole ? (T < st.n_sm ? (int)T : st.n_sm) : stream_grid(st, n_tiles, M);
+  if (grid > T * kc) grid = (int)(T * kc);
+  StreamArgs args{M, NP, n_tiles, row_groups, whole, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch, st.counters,
+                  status};
   k_gemm_stream<BN, MT, Epi><<<grid, UM_THREADS, smem, stream>>>(*ma, *mb0, *mb1, args, epi);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
   return 0;
 }
 
-// Row tiles the streaming kernel would use for M rows, or 0 when it cannot take the problem (more than 256 rows,
-// a tile too wide for two accumulators, or scratch / counters too small for its grid).
+// Row tiles per CTA the streaming kernel would use for M rows, or 0 when it cannot take the problem (a tile too wide
+// for the accumulators, scratch or counters too small for a split grid, too little shared memory).
 template <typename Epi>
 int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn) {
-  if (!st.use_stream || M > 2 * UM_BM || st.scratch == nullptr) return 0;
-  const int mt = M > UM_BM ? 2 : 1;
-  if (mt * bn > 512 || (mt == 2 && !st.stream_two_tiles)) return 0;
-  const int per_tile = Epi::kDual ? bn / 2 : bn;
-  const int n_tiles = (NP + per_tile - 1) / per_tile;
-  if (n_tiles > st.n_counters || stream_scratch_bytes(stream_grid(st, n_tiles, M), bn, mt) > st.scratch_bytes) return 0;
-  return stream_shape(st, M, bn, mt, K).stages >= 2 ? mt : 0;
+  if (!st.use_stream) return 0;
+  int mt;
+  if (M <= UM_BM) mt = 1;
+  else if (M <= 2 * UM_BM) mt = st.stream_two_tiles ? 2 : 0;
+  else if (st.stream_big_mt != 3) mt = st.stream_big_mt;   // 0 = leave large problems to the tiled kernel
+  else {
+    // 256 x 256 tiles (two row tiles per CTA) move a third less operand data through L2 per flop than 128 x 256 ones and
+    // measure about 12 % faster when both fill the SMs equally well; otherwise the fuller last wave wins
+    const int per_tile = Epi::kDual ? bn / 2 : bn;
+    const long n_tiles = (NP + per_tile - 1) / per_tile;
+    auto wave_eff = [&](int m) {
+      const long t = n_tiles * ((M + UM_BM * m - 1) / (UM_BM * m));
+      return (double)t / (double)((t + st.n_sm - 1) / st.n_sm * st.n_sm);
+    };
+    mt = (2 * bn <= 512 && 1.12 * wave_eff(2) > wave_eff(1)) ? 2 : 1;
+  }
+  if (mt == 0 || mt * bn > 512) return 0;
+  if (M <= UM_BM * mt) {                           // one row group: tiles may be split between CTAs
+    if (st.scratch == nullptr) return 0;
+    const int per_tile = Epi::kDual ? bn / 2 : bn;
+    const int n_tiles = (NP + per_tile - 1) / per_tile;
+    if (n_tiles > st.n_counters || stream_scratch_bytes(stream_grid(st, n_tiles, M), bn, mt) > st.scratch_bytes) return 0;
+  }
+  return stream_shape(st, stream_a_rows(M, mt), bn, mt, K).stages >= 2 ? mt : 0;
 }
 
 }  // namespace lsp

@@ -481,6 +481,8 @@ struct UmmaState {
   int skinny_bn = 128;             // tile width of plain epilogues in that regime
   int use_stream = 1;              // M <= 128: use the persistent weight-streaming kernel (gemm_stream.cuh)
   int stream_two_tiles = 1;        // ... also for 129..256 rows (two row tiles per CTA)
+  int stream_big_mt = 3;           // ... and for more rows: 1 or 2 row tiles per CTA, 3 = whichever fills the SMs better,
+                                   // 0 = leave those to the tiled kernel
   int stream_bn = 0;               // its tile width with one row tile (0 = automatic)
   int stream_bn2 = 0;              // ... and with two row tiles
   int stream_atoms = 0;            // K atoms per stage: 0 = two when stream_min_stages2 such stages fit, else 1 or 2 as given
@@ -620,7 +622,7 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
     const int num_kb = K / UM_BK;
     int max_bn = 256;
     if constexpr (std::is_same<Epi, EpiQKVRope<bf16>>::value) max_bn = 2 * epi.half;
-    if (M <= 2 * UM_BM) {
+    {
       // Tile width, from measurements on the LLaDA layer shapes at 2..256 rows: dual epilogues take 256 columns (128
       // pairs); plain ones take 128, which needs no K split with 96 tiles, except that a wide GEMM with at most 32
       // rows takes 256 (its partial tiles are small, and half as many MMA instructions are issued).  The rotary
@@ -630,8 +632,9 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
         box_rows = epi.half;
         sbn = (M <= 32) ? 256 : 128;
       }
+      if (M > 2 * UM_BM) sbn = 256;              // large problems: the widest MMA
       if (M <= UM_BM && st.stream_bn > 0) sbn = st.stream_bn;
-      if (M > UM_BM && st.stream_bn2 > 0) sbn = st.stream_bn2;
+      if (M > UM_BM && M <= 2 * UM_BM && st.stream_bn2 > 0) sbn = st.stream_bn2;
       if (box_rows > sbn / 2) sbn = 2 * box_rows;
       const int smt = stream_row_tiles<Epi>(st, M, NP, K, sbn);
       if (smt == 1) {
