@@ -275,12 +275,12 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         float4* slot_base = reinterpret_cast<float4*>(args.scratch + (size_t)(g * 2 + (seg == 0 ? 0 : 1)) * ROWS * BN);
 #pragma unroll 1
         for (int mt = 0; mt < MT; ++mt) {
-          const int m = mt * UM_BM + r_in;
+          const int m = mt * UM_BM + r_in;              // row within the row group
 #pragma unroll 1
           for (int c = 0; c < BN; c += 16) {
             float v[16];
             tc_ld16(t_row + mt * BN + c, v);
-            if (m < args.M) {
+            if (row0 + m < args.M) {
 #pragma unroll
               for (int i = 0; i < 4; ++i)
                 slot_base[(size_t)((c >> 4) * 4 + i) * ROWS + m] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
@@ -295,9 +295,9 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (threadIdx.x == 64) {
           const unsigned add = (unsigned)(seg_end - u);
-          const unsigned old = atomicAdd(args.counters + tile, add);
+          const unsigned old = atomicAdd(args.counters + tlin, add);
           const bool last = (old + add == (unsigned)args.kc);
-          if (last) args.counters[tile] = 0;          // ready for the next launch
+          if (last) args.counters[tlin] = 0;          // ready for the next launch
           *epi_flag = last ? 1u : 0u;
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -313,9 +313,10 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
           // plain epilogues: consecutive lanes take consecutive rows (coalesced reads of the partials); the reducing
           // epilogue keeps a row's chunks in neighbouring lanes so that they can be merged with shuffles
           const int ch = Epi::kReduce ? et % NCH : et / RPP, c = ch * 16;
-          for (int mm0 = 0; mm0 < args.M; mm0 += RPP) {
-            const int mm = mm0 + (Epi::kReduce ? et / NCH : et % RPP);
-            const bool valid = mm < args.M;
+          const int rows_here = min(ROWS, args.M - row0);           // rows of this row group
+          for (int mm0 = 0; mm0 < rows_here; mm0 += RPP) {
+            const int mm = mm0 + (Epi::kReduce ? et / NCH : et % RPP);   // row within the row group
+            const bool valid = mm < rows_here;
             float a0[16], a1[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
@@ -364,9 +365,9 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
               }
 #pragma unroll
               for (int o = 1; o < NCH; o <<= 1) red = top2_merge(red, top2_shfl_xor(red, o));
-              if (valid && ch == 0) epi.part[(size_t)mm * epi.n_tiles + tile] = red;
+              if (valid && ch == 0) epi.part[(size_t)(row0 + mm) * epi.n_tiles + tile] = red;
             } else {
-              if (valid && j0 + c < args.n_pairs) epi16(epi, mm, j0 + c, a0, a1);
+              if (valid && j0 + c < args.n_pairs) epi16(epi, row0 + mm, j0 + c, a0, a1);
             }
           }
         }
@@ -440,10 +441,10 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
   const int n_tiles = (NP + per_tile - 1) / per_tile;
   const int kc = K / (sh.atoms * UM_BK);
   const int row_groups = (M + UM_BM * MT - 1) / (UM_BM * MT);
-  // several row groups: whole tiles per CTA (the problem is large enough); one row group: K slices as stream_grid says
-  const int whole = row_groups > 1 ? 1 : 0;
+  // several row groups and at least as many tiles as SMs: whole tiles per CTA; else K slices as stream_grid says
   const long T = (long)n_tiles * row_groups;
-  int grid = whole ? (T < st.n_sm ? (int)T : st.n_sm) : stream_grid(st, n_tiles, M);
+  const int whole = (row_groups > 1 && T >= st.n_sm) ? 1 : 0;
+  int grid = whole ? st.n_sm : stream_grid(st, (int)T, M);
   if (grid > T * kc) grid = (int)(T * kc);
   StreamArgs args{M, NP, n_tiles, row_groups, whole, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch, st.counters,
                   status};
@@ -458,15 +459,15 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
 template <typename Epi>
 int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn) {
   if (!st.use_stream) return 0;
+  const int per_tile = Epi::kDual ? bn / 2 : bn;
+  const long n_tiles = (NP + per_tile - 1) / per_tile;
   int mt;
   if (M <= UM_BM) mt = 1;
-  else if (M <= 2 * UM_BM) mt = st.stream_two_tiles ? 2 : 0;
+  else if (M <= 2 * UM_BM) mt = st.stream_two_tiles == 1 ? 2 : (st.stream_two_tiles == 2 ? 1 : 0);
   else if (st.stream_big_mt != 3) mt = st.stream_big_mt;   // 0 = leave large problems to the tiled kernel
   else {
     // 256 x 256 tiles (two row tiles per CTA) move a third less operand data through L2 per flop than 128 x 256 ones and
     // measure about 12 % faster when both fill the SMs equally well; otherwise the fuller last wave wins
-    const int per_tile = Epi::kDual ? bn / 2 : bn;
-    const long n_tiles = (NP + per_tile - 1) / per_tile;
     auto wave_eff = [&](int m) {
       const long t = n_tiles * ((M + UM_BM * m - 1) / (UM_BM * m));
       return (double)t / (double)((t + st.n_sm - 1) / st.n_sm * st.n_sm);
@@ -474,11 +475,12 @@ int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn) {
     mt = (2 * bn <= 512 && 1.12 * wave_eff(2) > wave_eff(1)) ? 2 : 1;
   }
   if (mt == 0 || mt * bn > 512) return 0;
-  if (M <= UM_BM * mt) {                           // one row group: tiles may be split between CTAs
-    if (st.scratch == nullptr) return 0;
-    const int per_tile = Epi::kDual ? bn / 2 : bn;
-    const int n_tiles = (NP + per_tile - 1) / per_tile;
-    if (n_tiles > st.n_counters || stream_scratch_bytes(stream_grid(st, n_tiles, M), bn, mt) > st.scratch_bytes) return 0;
+  const int row_groups = (M + UM_BM * mt - 1) / (UM_BM * mt);
+  const long T = n_tiles * row_groups;
+  if (!(row_groups > 1 && T >= st.n_sm)) {         // tiles may be split between CTAs: scratch and counters
+    if (st.scratch == nullptr || T > st.n_counters ||
+        stream_scratch_bytes(stream_grid(st, (int)T, M), bn, mt) > st.scratch_bytes)
+      return 0;
   }
   return stream_shape(st, stream_a_rows(M, mt), bn, mt, K).stages >= 2 ? mt : 0;
 }

@@ -480,7 +480,7 @@ struct UmmaState {
   int skinny_min_stages = 3;       // ... provided each still gets this many pipeline stages
   int skinny_bn = 128;             // tile width of plain epilogues in that regime
   int use_stream = 1;              // M <= 128: use the persistent weight-streaming kernel (gemm_stream.cuh)
-  int stream_two_tiles = 1;        // ... also for 129..256 rows (two row tiles per CTA)
+  int stream_two_tiles = 1;        // ... also for 129..256 rows: 1 = two row tiles per CTA, 2 = two row groups, 0 = no
   int stream_big_mt = 3;           // ... and for more rows: 1 or 2 row tiles per CTA, 3 = whichever fills the SMs better,
                                    // 0 = leave those to the tiled kernel
   int stream_bn = 0;               // its tile width with one row tile (0 = automatic)
@@ -632,7 +632,7 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
         box_rows = epi.half;
         sbn = (M <= 32) ? 256 : 128;
       }
-      if (M > 2 * UM_BM) sbn = 256;              // large problems: the widest MMA
+      if (M > 2 * UM_BM || (M > UM_BM && st.stream_two_tiles == 2)) sbn = 256;   // several row groups: the widest MMA
       if (M <= UM_BM && st.stream_bn > 0) sbn = st.stream_bn;
       if (M > UM_BM && M <= 2 * UM_BM && st.stream_bn2 > 0) sbn = st.stream_bn2;
       if (box_rows > sbn / 2) sbn = 2 * box_rows;
