@@ -134,7 +134,9 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * 20 = its tile width for those (0 = automatic, 64, 128 or 256), 21 = 64-element K atoms per pipeline stage (0 = automatic, 1, 2),
  * 22 = fewest two-atom stages the automatic choice accepts, 23 = its tile width for up to 128 rows (0 = automatic,
  * 64, 128 or 256), 24 = row tiles per CTA it uses for more than 256 rows (1, 2,
- * 3 = automatic, default; 0 = the tiled kernel takes those). */
+ * 3 = automatic, default; 0 = the tiled kernel takes those), 25 = launch the step's kernels with programmatic dependent
+ * launch, so that each kernel's set-up overlaps its predecessor's tail (1) or plainly (0, default: the step is bound by
+ * kernel time, not by launch gaps, and the overlap measured no gain). */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

@@ -58,6 +58,7 @@ __global__ void __launch_bounds__(128) k_attn_mma(const bf16* __restrict__ q, co
   constexpr int LD = DH + 8;            // padded row (elements): 16-byte shift per row, conflict-free ldmatrix
   constexpr int CPR = DH / 8;           // 16-byte chunks per row
   extern __shared__ __align__(16) uint8_t attn_smem[];
+  pdl_begin();
   bf16* Qs = reinterpret_cast<bf16*>(attn_smem);
   bf16* Ks = Qs + AM_BM * LD;           // [2][AM_BN][LD]
   bf16* Vs = Ks + 2 * AM_BN * LD;       // [2][AM_BN][LD]

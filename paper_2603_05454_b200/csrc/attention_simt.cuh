@@ -21,6 +21,7 @@ __global__ void __launch_bounds__(128) k_attn_simt(const T* __restrict__ q, cons
   __shared__ float Qs[AS_BQ][DH];
   __shared__ float Ks[AS_BK][DH + 1];
   __shared__ float Vs[AS_BK][DH];
+  pdl_begin();
   const int b = blockIdx.z, h = blockIdx.y;
   const int r0 = sd.row_off[b];
   const int Qn = sd.row_off[b + 1] - r0;

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace lsp {
 
 typedef __nv_bfloat16 bf16;
@@ -77,6 +79,33 @@ __device__ __forceinline__ float warp_min(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
+}
+
+// Programmatic dependent launch.  Every kernel of a step is launched with the programmatic-serialisation attribute
+// (launch_k below): it lets the next kernel's blocks be scheduled, and run their set-up, while the previous kernel
+// drains.  pdl_begin() is the first statement of every kernel: it releases the following launch at once (that launch
+// waits itself) and then waits until the preceding kernel has completed and its writes are visible.  Kernels with a
+// set-up that touches no global memory call pdl_release() first and pdl_wait() after the set-up.  Both are no-ops in a
+// kernel launched without the attribute.
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_begin() { pdl_release(); pdl_wait(); }
+
+// Launches kernel(args...) on stream; pdl = 1 adds the programmatic-serialisation attribute.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(int pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                            Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
 }
 
 // Per-step descriptor the host uploads before each pass (int32 arrays of batch+1 entries each).

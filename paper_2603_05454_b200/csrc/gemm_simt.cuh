@@ -25,6 +25,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const T* __restrict__ A, cons
   __shared__ float As[SG_BK][SG_BM + 4];
   __shared__ float B0s[SG_BK][SG_BN + 4];
   __shared__ float B1s[Epi::kDual ? SG_BK : 1][SG_BN + 4];
+  pdl_begin();
   const int t = threadIdx.x;
   const int m0 = blockIdx.y * SG_BM, j0 = blockIdx.x * SG_BN;
   const int lrow = t >> 2, lk = (t & 3) * 4;

@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
 k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
               const __grid_constant__ CUtensorMap map_b1, StreamArgs args, Epi epi) {
   extern __shared__ uint8_t smem_raw[];
+  pdl_release();
   constexpr int HALF = BN / 2;
   constexpr int B_HALF_ATOM = HALF * 128;               // bytes of one half-tile atom (64 K elements)
   constexpr int B_ATOM = BN * 128;
@@ -110,6 +111,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();          // barriers and tensor memory are set up; from here on the kernel reads what its predecessor wrote
 
   const int G = gridDim.x, g = blockIdx.x;
   const int RG = args.row_groups;
@@ -448,8 +450,8 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
   if (grid > T * kc) grid = (int)(T * kc);
   StreamArgs args{M, NP, n_tiles, row_groups, whole, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch, st.counters,
                   status};
-  k_gemm_stream<BN, MT, Epi><<<grid, UM_THREADS, smem, stream>>>(*ma, *mb0, *mb1, args, epi);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_k(st.pdl, k_gemm_stream<BN, MT, Epi>, dim3(grid), dim3(UM_THREADS), smem, stream, *ma, *mb0, *mb1, args, epi);
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
   return 0;
 }

@@ -293,6 +293,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
 k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
             const __grid_constant__ CUtensorMap map_b1, UmmaArgs args, Epi epi) {
   extern __shared__ uint8_t smem_raw[];
+  pdl_release();
   constexpr int B_HALF_BYTES = (BN / 2) * UM_BK * 2;
   constexpr int HALF = BN / 2;
   const int A_BYTES = args.a_rows * UM_BK * 2;             // a multiple of 1024: the weight tile stays swizzle-aligned
@@ -345,6 +346,7 @@ k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();          // barriers and tensor memory are set up; from here on the kernel reads what its predecessor wrote
   const int kb0 = blockIdx.z * args.kb_per_split;
   const int num_kb = min(args.kb_per_split, args.num_kb - kb0);
 
@@ -479,6 +481,7 @@ struct UmmaState {
   int skinny_ctas_per_sm = 2;      // co-resident CTAs a weight-streaming (M <= 128) launch aims for
   int skinny_min_stages = 3;       // ... provided each still gets this many pipeline stages
   int skinny_bn = 128;             // tile width of plain epilogues in that regime
+  int pdl = 0;                     // launch with the programmatic-serialisation attribute (measured: no gain, off)
   int use_stream = 1;              // M <= 128: use the persistent weight-streaming kernel (gemm_stream.cuh)
   int stream_two_tiles = 1;        // ... also for 129..256 rows: 1 = two row tiles per CTA, 2 = two row groups, 0 = no
   int stream_big_mt = 3;           // ... and for more rows: 1 or 2 row tiles per CTA, 3 = whichever fills the SMs better,
@@ -574,8 +577,8 @@ int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W
   if (m_fast) grid = dim3(grid.y, grid.x);
   grid.z = splits;
   UmmaArgs args{M, NP, K, num_kb, stages, plan.a_rows, m_fast, splits, kb_per_split, st.scratch, st.counters, status};
-  k_gemm_umma<BN, Epi><<<grid, UM_THREADS, smem, stream>>>(*ma, *mb0, *mb1, args, epi);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = launch_k(st.pdl, k_gemm_umma<BN, Epi>, grid, dim3(UM_THREADS), smem, stream, *ma, *mb0, *mb1, args, epi);
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
   return 0;
 }

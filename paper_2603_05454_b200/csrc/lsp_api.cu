@@ -34,7 +34,7 @@ struct lsp_ctx {
   int max_batch = 0, max_len = 0, max_rows = 0;
   size_t esz = 0;
   cudaStream_t stream = nullptr;
-  int gemm_impl = 1, attn_impl = 1, timing = 0, async_ops = 0, op_repeat = 1, op_rotate = 1;
+  int gemm_impl = 1, attn_impl = 1, timing = 0, async_ops = 0, op_repeat = 1, op_rotate = 1, pdl = 0;
   // workspace carve (device)
   char *X = nullptr, *Nrm = nullptr, *Qb = nullptr, *Att = nullptr, *Hf = nullptr, *stage = nullptr;
   Top2* part = nullptr;
@@ -224,8 +224,7 @@ int run_gemm(lsp_ctx* c, const T* A, const T* W0, const T* W1, int M, int NP, in
   }
 #endif
   dim3 grid((NP + SG_BN - 1) / SG_BN, (M + SG_BM - 1) / SG_BM);
-  k_gemm_simt<T, Epi><<<grid, 256, 0, c->stream>>>(A, W0, W1, M, NP, K, epi);
-  CU(cudaGetLastError());
+  CU(launch_k(c->pdl, k_gemm_simt<T, Epi>, grid, dim3(256), 0, c->stream, A, W0, W1, M, NP, K, epi));
   return LSP_OK;
 }
 
@@ -264,13 +263,13 @@ ScanParams scan_params(const lsp_ctx* c) {
 // merge partials -> scores, scan, copy the scan outputs to the pinned mirror (async)
 int run_merge_scan(lsp_ctx* c, int rows, int n_tiles, const int* d_seq_off, int batch) {
   if (rows > 0) {
-    k_merge_partials<<<(rows + 3) / 4, 128, 0, c->stream>>>(c->part, n_tiles, rows, c->yhat, c->pmax, c->margin);
-    CU(cudaGetLastError());
+    CU(launch_k(c->pdl, k_merge_partials, dim3((rows + 3) / 4), dim3(128), 0, c->stream, (const Top2*)c->part, n_tiles, rows, c->yhat,
+                c->pmax, c->margin));
   }
   const float* score = c->s.score == 1 ? c->margin : c->pmax;
   int* o = c->d_scan;
   const int mb = c->max_batch;
-  k_lsp_scan<<<batch, 32, 0, c->stream>>>(score, c->yhat, c->margin, d_seq_off, scan_params(c), o, o + mb,
+  launch_k(c->pdl, k_lsp_scan, dim3(batch), dim3(32), 0, c->stream, score, c->yhat, c->margin, d_seq_off, scan_params(c), o, o + mb,
                                           (uint32_t*)(o + 2 * mb), (float*)(o + 3 * mb));
   CU(cudaGetLastError());
   CU(cudaMemcpyAsync(c->h_scan, c->d_scan, 4 * (size_t)mb * 4, cudaMemcpyDeviceToHost, c->stream));
@@ -324,7 +323,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   T* Att = (T*)c->Att;
   T* Hf = (T*)c->Hf;
   seg_begin(c, CLS_MISC);
-  k_assemble_embed<T><<<M, 128, 0, c->stream>>>(sd, B, c->tokens, c->tok_stride, m.mask_id, (const T*)c->embed, d, X,
+  launch_k(c->pdl, k_assemble_embed<T>, dim3(M), dim3(128), 0, c->stream, sd, B, c->tokens, c->tok_stride, m.mask_id, (const T*)c->embed, d, X,
                                                c->row_seq, c->row_pos, c->head_src);
   seg_end(c);
   count_launch(c, CLS_MISC);
@@ -338,7 +337,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
     const T* cK = (const T*)c->kv_cache + (size_t)(2 * l) * cplane;
     const T* cV = cK + cplane;
     seg_begin(c, CLS_MISC);
-    k_rmsnorm<T><<<M, 256, 0, c->stream>>>(X, (const T*)c->attn_norm[l], Nrm, nullptr, d, m.rms_eps);
+    launch_k(c->pdl, k_rmsnorm<T>, dim3(M), dim3(256), 0, c->stream, X, (const T*)c->attn_norm[l], Nrm, nullptr, d, m.rms_eps);
     seg_end(c);
     count_launch(c, CLS_MISC);
     CU(cudaGetLastError());
@@ -365,21 +364,19 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
           dim3 g2((maxQ * G + AM_BM - 1) / AM_BM, m.n_kv_heads, B);
           const float sl2 = scale * 1.4426950408889634f;
           if (dh == 128)
-            k_attn_mma<128><<<g2, 128, attn_mma_smem_bytes<128>(), c->stream>>>(
-                Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
+            launch_k(c->pdl, k_attn_mma<128>, dim3(g2), dim3(128), attn_mma_smem_bytes<128>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
           else
-            k_attn_mma<64><<<g2, 128, attn_mma_smem_bytes<64>(), c->stream>>>(
-                Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
+            launch_k(c->pdl, k_attn_mma<64>, dim3(g2), dim3(128), attn_mma_smem_bytes<64>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
           done = true;
         }
       }
       dim3 grid((maxQ + AS_BQ - 1) / AS_BQ, m.n_heads, B);
       if (done) {
       } else if (dh == 128)
-        k_attn_simt<T, 128><<<grid, 128, 0, c->stream>>>(Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
+        launch_k(c->pdl, k_attn_simt<T, 128>, dim3(grid), dim3(128), 0, c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
                                                          (size_t)c->max_len * kvd, scale);
       else
-        k_attn_simt<T, 64><<<grid, 128, 0, c->stream>>>(Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
+        launch_k(c->pdl, k_attn_simt<T, 64>, dim3(grid), dim3(128), 0, c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
                                                         (size_t)c->max_len * kvd, scale);
       seg_end(c);
       CU(cudaGetLastError());
@@ -390,7 +387,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
       if (rc) return rc;
     }
     seg_begin(c, CLS_MISC);
-    k_rmsnorm<T><<<M, 256, 0, c->stream>>>(X, (const T*)c->ffn_norm[l], Nrm, nullptr, d, m.rms_eps);
+    launch_k(c->pdl, k_rmsnorm<T>, dim3(M), dim3(256), 0, c->stream, X, (const T*)c->ffn_norm[l], Nrm, nullptr, d, m.rms_eps);
     seg_end(c);
     count_launch(c, CLS_MISC);
     CU(cudaGetLastError());
@@ -407,7 +404,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   }
   // masked rows only: final norm (gathered), fused head, merge, scan
   seg_begin(c, CLS_MISC);
-  k_rmsnorm<T><<<Mh, 256, 0, c->stream>>>(X, (const T*)c->final_norm, Nrm, c->head_src, d, m.rms_eps);
+  launch_k(c->pdl, k_rmsnorm<T>, dim3(Mh), dim3(256), 0, c->stream, X, (const T*)c->final_norm, Nrm, c->head_src, d, m.rms_eps);
   seg_end(c);
   count_launch(c, CLS_MISC);
   CU(cudaGetLastError());
@@ -617,6 +614,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   else if (key == 10) c->umma.target_ctas = value;
   else if (key == 11) c->umma.max_stages = value < 1 ? 1 : (value > UM_MAX_STAGES ? UM_MAX_STAGES : value);
   else if (key == 12) c->umma.allow_split = value;
+  else if (key == 25) { c->pdl = value ? 1 : 0; c->umma.pdl = c->pdl; }
   else if (key == 16) c->umma.use_stream = value;
   else if (key == 17) c->umma.stream_grid_mode = value;
   else if (key == 18) c->umma.stream_even_max_rows = value;
@@ -697,7 +695,7 @@ int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
   if (chunks > 64) chunks = 64;
   dim3 grid(chunks, m.n_layers * 2, B);
   seg_begin(c, CLS_COMMIT);
-  k_commit_append<<<grid, 256, 0, c->stream>>>(desc_of(c), (const uint4*)c->stage, (uint4*)c->kv_cache,
+  launch_k(c->pdl, k_commit_append, dim3(grid), dim3(256), 0, c->stream, desc_of(c), (const uint4*)c->stage, (uint4*)c->kv_cache,
                                                stage_plane_v4, cache_plane_v4, cache_seq_v4, row_v4, c->yhat,
                                                c->tokens, c->tok_stride);
   seg_end(c);
@@ -810,7 +808,7 @@ int lsp_scan(lsp_ctx* c, const float* score, const int32_t* yhat, const float* m
   c->proposed = false;
   int* o = c->d_scan;
   const int mb = c->max_batch;
-  k_lsp_scan<<<batch, 32, 0, c->stream>>>(score, yhat, margin, c->d_desc + 4 * (c->max_batch + 1), scan_params(c), o,
+  launch_k(c->pdl, k_lsp_scan, dim3(batch), dim3(32), 0, c->stream, score, yhat, margin, c->d_desc + 4 * (c->max_batch + 1), scan_params(c), o,
                                           o + mb, (uint32_t*)(o + 2 * mb), (float*)(o + 3 * mb));
   CU(cudaGetLastError());
   CU(cudaMemcpyAsync(c->h_scan, c->d_scan, 4 * (size_t)mb * 4, cudaMemcpyDeviceToHost, c->stream));

@@ -14,6 +14,7 @@ __global__ void k_assemble_embed(StepDesc sd, int batch, const int32_t* __restri
                                  int mask_id, const T* __restrict__ embed, int d, T* __restrict__ X,
                                  int* __restrict__ row_seq, int* __restrict__ row_pos,
                                  int* __restrict__ head_src) {
+  pdl_begin();
   const int r = blockIdx.x;
   int b = 0;
   while (b + 1 < batch && r >= sd.row_off[b + 1]) ++b;
@@ -67,6 +68,7 @@ __global__ void __launch_bounds__(RN_THREADS) k_rmsnorm(const T* __restrict__ x,
                                                        const int* __restrict__ src_rows, int d, float eps) {
   constexpr int E = Vec16<T>::N;                 // elements per 16-byte vector
   __shared__ float red[RN_THREADS / 32];
+  pdl_begin();
   const int r = blockIdx.x;
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)(src_rows ? src_rows[r] : r) * d);
   const uint4* gr = reinterpret_cast<const uint4*>(g);
@@ -133,6 +135,7 @@ __global__ void __launch_bounds__(RN_THREADS) k_rmsnorm(const T* __restrict__ x,
 // ---------------------------------------------------------------------------------------------
 __global__ void k_merge_partials(const Top2* __restrict__ part, int n_tiles, int rows, int32_t* __restrict__ yhat,
                                  float* __restrict__ pmax, float* __restrict__ margin) {
+  pdl_begin();
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= rows) return;
   const int lane = threadIdx.x & 31;
@@ -171,6 +174,7 @@ __global__ void k_lsp_scan(const float* __restrict__ score, const int32_t* __res
                            const float* __restrict__ margin, const int* __restrict__ seq_off, ScanParams p,
                            int32_t* __restrict__ o_run, int32_t* __restrict__ o_commit, uint32_t* __restrict__ o_flags,
                            float* __restrict__ o_tau) {
+  pdl_begin();
   const int b = blockIdx.x;
   const int lane = threadIdx.x;
   const int base = seq_off[b];
@@ -275,6 +279,7 @@ __global__ void k_commit_append(StepDesc sd, const uint4* __restrict__ stage, ui
                                 size_t cache_seq_v4,     // uint4 per sequence inside a cache plane
                                 int row_v4,              // uint4 per row (n_kv_heads * head_dim * sizeof(T) / 16)
                                 const int32_t* __restrict__ yhat, int32_t* __restrict__ tokens, int tok_stride) {
+  pdl_begin();
   const int b = blockIdx.z;
   const int plane = blockIdx.y;
   const int pend = sd.pend[b];

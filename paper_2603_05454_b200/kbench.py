@@ -98,7 +98,7 @@ def _fast_weights(sh):
                              w_down=rnd(d, f), attn_norm=one(), ffn_norm=one()) for _ in range(sh.n_layers)])
 
 
-def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False):
+def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False, opts=()):
     """Per-class kernel times of a decode.  layers > 0 cuts the model to its first layers, max_passes > 0 stops each
     decode after that many denoiser passes (both are profiling aids: fewer launches, same kernels and row counts)."""
     wl = S.config(name)
@@ -109,6 +109,8 @@ def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False):
     w = _fast_weights(sh) if fast_init else S.make_weights(sh, 0, device=DEV)
     dec = LSPDecoder(sh, w, SchedCfg(tau=wl.tau, delim_bitmap=S.delimiter_bitmap(sh.vocab, *wl.delim).to(DEV)), B, P + G,
                      device=DEV)
+    for k, v in opts:
+        dec.set_option(k, v)
     tokens = torch.zeros(B, P + G, dtype=torch.int32, device=DEV)
     tokens[:, :P] = S.make_prompt(B, P, sh, 100).to(DEV)
 
@@ -173,7 +175,7 @@ def main():
         for m in a.M:
             print(json.dumps(bench_head(m, a.V, a.d, a.reps)), flush=True)
     else:
-        print(json.dumps(bench_decode(a.workload, 1, a.layers, a.max_passes, a.fast_init)), flush=True)
+        print(json.dumps(bench_decode(a.workload, 1, a.layers, a.max_passes, a.fast_init, a.opt)), flush=True)
 
 
 if __name__ == "__main__":
