@@ -136,7 +136,8 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * 64, 128 or 256), 24 = row tiles per CTA it uses for more than 256 rows (1, 2,
  * 3 = automatic, default; 0 = the tiled kernel takes those), 25 = launch the step's kernels with programmatic dependent
  * launch, so that each kernel's set-up overlaps its predecessor's tail (1) or plainly (0, default: the step is bound by
- * kernel time, not by launch gaps, and the overlap measured no gain). */
+ * kernel time, not by launch gaps, and the overlap measured no gain), 26 = MMA-issuing warps of the persistent kernel with one
+ * row tile per CTA (1, default, or 2). */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

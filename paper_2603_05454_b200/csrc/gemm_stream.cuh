@@ -19,10 +19,10 @@
 //   * a tile that spans several CTAs is finished by the CTA that arrives last at the tile's counter: every
 //     contributor writes its fp32 partial tile to scratch, and the finisher sums all of them in CTA order (the same
 //     order whoever finishes, so results are deterministic) before running the fused epilogue.
-// Tile width: one tcgen05.mma with M = 128 occupies the tensor pipe for about 150 cycles whatever its N (measured
-// for N = 16..256), so a narrow tile does not make the instruction cheaper; 256-column tiles halve the instruction
-// count per weight byte against 128-column ones and keep the MMA time below the weight-streaming time.
-// Warp roles as in gemm_umma.cuh: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = epilogue.
+// Tile width: measured per shape and row count (see umma_gemm): 128 columns for plain epilogues in the streaming
+// regime (no K split needed with 96 tiles), 256 for dual epilogues and for every problem with several row groups.
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = epilogue, warp 6 = second MMA
+// issuer (see the note on issue rate in the kernel).
 // Every wait is bounded; on expiry the kernel records (code, site) in the status word, drains and returns.
 #pragma once
 #include "gemm_umma.cuh"
@@ -57,8 +57,10 @@ __device__ __forceinline__ long st_first_unit(long U, int G, int g) { return U *
 // CTA that owns unit u
 __device__ __forceinline__ int st_owner(long U, int G, long u) { return (int)(((u + 1) * G + U - 1) / U) - 1; }
 
-template <int BN, int MT, typename Epi>
-__global__ void __launch_bounds__(UM_THREADS, 1)
+constexpr int ST_THREADS = 224;            // warp 0 producer, warps 1 and 6 MMA issuers, warps 2..5 epilogue
+
+template <int BN, int MT, int NI, typename Epi>
+__global__ void __launch_bounds__(ST_THREADS, 1)
 k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
               const __grid_constant__ CUtensorMap map_b1, StreamArgs args, Epi epi) {
   extern __shared__ uint8_t smem_raw[];
@@ -67,8 +69,17 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   constexpr int B_HALF_ATOM = HALF * 128;               // bytes of one half-tile atom (64 K elements)
   constexpr int B_ATOM = BN * 128;
   constexpr int ROWS = UM_BM * MT;                        // accumulator rows
-  constexpr int NBUF = (2 * MT * BN <= 512) ? 2 : 1;      // accumulator sets in tensor memory
-  constexpr uint32_t TMEM_COLS = NBUF * MT * BN;
+  // In an isolated probe one thread issues a tcgen05.mma about every 150 cycles whatever the instruction's N, and two
+  // issuing threads in different warps double that rate.  NI = 2 therefore lets two warps share the issue without sharing
+  // an accumulator: with two row tiles each takes one; with one row tile they take alternate K steps into accumulators of
+  // their own (ACC = 2), which the epilogue adds.  In this kernel the issue rate turned out not to be the limit (the
+  // operand stream is): NI = 2 measures the same as NI = 1 at every shape, so one row tile uses NI = 1 by default.
+  static_assert(NI == 1 || NI == 2, "one or two MMA issuers");
+  static_assert(MT == 1 || NI == 2, "two row tiles are issued by two warps");
+  constexpr int ACC = (MT == 1 && NI == 2) ? 2 : 1;       // accumulators per row tile
+  constexpr int SET_COLS = MT * ACC * BN;                 // columns of one accumulator set
+  constexpr int NBUF = (2 * SET_COLS <= 512) ? 2 : 1;     // accumulator sets in tensor memory
+  constexpr uint32_t TMEM_COLS = NBUF * SET_COLS;
   const int A_ATOM = args.a_rows * 128;
   const int AT = args.atoms;
   const int STAGE_BYTES = AT * (A_ATOM + B_ATOM);
@@ -90,10 +101,10 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
+      mbar_init(empty_bar(s), NI);          // every issuer commits the stage
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(accf_bar(b), 1);
+      mbar_init(accf_bar(b), NI);           // ... and the accumulator set
       mbar_init(acce_bar(b), 4);
     }
     *abort_flag = 0;
@@ -170,9 +181,10 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         mbar_wait(full_bar((int)(it % S)), (uint32_t)(it / S) & 1u, &no_abort);
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+  } else if (warp == 1 || warp == 6) {
+    // ---------------- MMA issuers ----------------
+    const int is = warp == 1 ? 0 : 1;                   // issuer index
+    if (lane == 0 && is < NI) {
       constexpr uint32_t idesc = make_idesc(BN);
       int seg = 0;
       bool ok = true;
@@ -189,7 +201,8 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
           break;
         }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
+        // this issuer's accumulator: row tile `is` (two row tiles) or K-parity accumulator `is` (one row tile)
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * SET_COLS + (NI == 2 ? is * BN : 0));
         bool first = true;
         for (; u < seg_end; ++u) {
           if (!mbar_wait(full_bar(s), ph, abort_flag)) {
@@ -201,14 +214,13 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
           const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
           const uint32_t sb = sa + AT * A_ATOM;
           for (int j = 0; j < AT; ++j) {
-            const uint64_t da = make_smem_desc(sa + j * A_ATOM);
+            // row tile 1 starts 128 rows = 16 KB (1024 descriptor units) further into the activation atom
+            const uint64_t da = make_smem_desc(sa + j * A_ATOM) + (uint64_t)((MT == 2 && is == 1) ? 1024 : 0);
             const uint64_t db = make_smem_desc(sb + j * B_ATOM);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-#pragma unroll
-              for (int mt = 0; mt < MT; ++mt)   // row tile mt starts 128 rows = 16 KB further into the activation atom
-                tc_mma_f16(d_tmem + (uint32_t)(mt * BN), da + (uint64_t)(mt * 1024 + 2 * k), db + (uint64_t)(2 * k), idesc,
-                           first ? 0u : 1u);
+              if (MT == 1 && NI == 2 && (k & 1) != is) continue;       // alternate K steps
+              tc_mma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, first ? 0u : 1u);
               first = false;
             }
           }
@@ -240,7 +252,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         break;
       }
       tc_fence_after();
-      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * MT * BN);
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * SET_COLS);
       const int j0 = tile * CH;
       if (whole) {
         // the accumulator is complete in tensor memory: each thread owns one row of every row tile
@@ -251,8 +263,19 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
 #pragma unroll 1
           for (int c = 0; c < CH; c += 16) {
             float a0[16], a1[16];
-            tc_ld16(t_row + mt * BN + c, a0);
-            if (Epi::kDual) tc_ld16(t_row + mt * BN + HALF + c, a1);
+            tc_ld16(t_row + mt * ACC * BN + c, a0);
+            if (Epi::kDual) tc_ld16(t_row + mt * ACC * BN + HALF + c, a1);
+            if constexpr (ACC == 2) {               // add the second K-parity accumulator
+              float b0[16];
+              tc_ld16(t_row + BN + c, b0);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) a0[i] += b0[i];
+              if (Epi::kDual) {
+                tc_ld16(t_row + BN + HALF + c, b0);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) a1[i] += b0[i];
+              }
+            }
             if constexpr (Epi::kReduce) {
 #pragma unroll
               for (int i = 0; i < 16; ++i) {
@@ -281,7 +304,13 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
 #pragma unroll 1
           for (int c = 0; c < BN; c += 16) {
             float v[16];
-            tc_ld16(t_row + mt * BN + c, v);
+            tc_ld16(t_row + mt * ACC * BN + c, v);
+            if constexpr (ACC == 2) {
+              float b0[16];
+              tc_ld16(t_row + BN + c, b0);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) v[i] += b0[i];
+            }
             if (row0 + m < args.M) {
 #pragma unroll
               for (int i = 0; i < 4; ++i)
@@ -421,7 +450,7 @@ inline StreamShape stream_shape(const UmmaState& st, int a_rows, int bn, int mt,
 // Activation box rows: all rows (rounded up to 8) when they fit one group of 128 mt rows, else a full group.
 inline int stream_a_rows(int M, int mt) { return M <= UM_BM * mt ? (M + 7) / 8 * 8 : UM_BM * mt; }
 
-template <int BN, int MT, typename Epi>
+template <int BN, int MT, int NI, typename Epi>
 int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
                   int n_rows_w, const Epi& epi, unsigned* status, int box_rows) {
   const StreamShape sh = stream_shape(st, stream_a_rows(M, MT), BN, MT, K);
@@ -429,7 +458,7 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
   const size_t smem = (size_t)sh.stages * sh.stage_bytes + sh.aux;
   static bool attr_set = false;   // per instantiation
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(k_gemm_stream<BN, MT, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, st.max_smem);
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_stream<BN, MT, NI, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, st.max_smem);
     if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -3; }
     attr_set = true;
   }
@@ -450,7 +479,7 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
   if (grid > T * kc) grid = (int)(T * kc);
   StreamArgs args{M, NP, n_tiles, row_groups, whole, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch, st.counters,
                   status};
-  cudaError_t e = launch_k(st.pdl, k_gemm_stream<BN, MT, Epi>, dim3(grid), dim3(UM_THREADS), smem, stream, *ma, *mb0, *mb1, args, epi);
+  cudaError_t e = launch_k(st.pdl, k_gemm_stream<BN, MT, NI, Epi>, dim3(grid), dim3(ST_THREADS), smem, stream, *ma, *mb0, *mb1, args, epi);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
   return 0;

@@ -483,6 +483,7 @@ struct UmmaState {
   int skinny_bn = 128;             // tile width of plain epilogues in that regime
   int pdl = 0;                     // launch with the programmatic-serialisation attribute (measured: no gain, off)
   int use_stream = 1;              // M <= 128: use the persistent weight-streaming kernel (gemm_stream.cuh)
+  int stream_issuers = 1;          // MMA-issuing warps with one row tile per CTA (two row tiles always use two); measured: no gain from 2
   int stream_two_tiles = 1;        // ... also for 129..256 rows: 1 = two row tiles per CTA, 2 = two row groups, 0 = no
   int stream_big_mt = 3;           // ... and for more rows: 1 or 2 row tiles per CTA, 3 = whichever fills the SMs better,
                                    // 0 = leave those to the tiled kernel
@@ -584,9 +585,31 @@ int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W
 }
 
 template <typename Epi> int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn);
-template <int BN, int MT, typename Epi>
+template <int BN, int MT, int NI, typename Epi>
 int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
                   int n_rows_w, const Epi& epi, unsigned* status, int box_rows);
+
+// Instantiation choice for the streaming kernel: tile width 128 or 256, one or two row tiles, one or two MMA issuers
+// (two row tiles always have two).
+template <typename Epi>
+int stream_dispatch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
+                    int n_rows_w, const Epi& epi, unsigned* status, int box_rows, int bn, int mt, int ni) {
+#define LSP_STREAM_CASE(BN_, MT_, NI_) \
+  if (bn == BN_ && mt == MT_ && ni == NI_) \
+    return stream_launch<BN_, MT_, NI_, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows)
+  if (mt == 2) ni = 2;
+  LSP_STREAM_CASE(256, 1, 1);
+  LSP_STREAM_CASE(256, 1, 2);
+  LSP_STREAM_CASE(256, 2, 2);
+  if constexpr (!Epi::kReduce) {
+    LSP_STREAM_CASE(128, 1, 1);
+    LSP_STREAM_CASE(128, 1, 2);
+    LSP_STREAM_CASE(128, 2, 2);
+  }
+#undef LSP_STREAM_CASE
+  st.err = "no streaming-kernel instantiation for this tile shape";
+  return -7;
+}
 
 // Tile-width and split-K choice.
 //  * Problems with at most 256 activation rows go to the persistent weight-streaming kernel (gemm_stream.cuh) when it
@@ -609,10 +632,11 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
     while (plan.a_rows < M) plan.a_rows *= 2;
   }
   if constexpr (Epi::kReduce) {
-    switch (stream_row_tiles<Epi>(st, M, NP, K, UM_HEAD_BN)) {
-      case 1: return stream_launch<UM_HEAD_BN, 1, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 0);
-      case 2: return stream_launch<UM_HEAD_BN, 2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 0);
-      default: break;
+    {
+      const int smt = stream_row_tiles<Epi>(st, M, NP, K, UM_HEAD_BN);
+      if (smt > 0)
+        return stream_dispatch<Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 0, UM_HEAD_BN, smt,
+                                    st.stream_issuers);
     }
     if (mt == 1 && st.skinny_ctas_per_sm > 1) {
       const int stage = plan.a_rows * UM_BK * 2 + UM_HEAD_BN * UM_BK * 2;
@@ -640,21 +664,9 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
       if (M > UM_BM && M <= 2 * UM_BM && st.stream_bn2 > 0) sbn = st.stream_bn2;
       if (box_rows > sbn / 2) sbn = 2 * box_rows;
       const int smt = stream_row_tiles<Epi>(st, M, NP, K, sbn);
-      if (smt == 1) {
-        switch (sbn) {
-          case 256: return stream_launch<256, 1, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
-          case 128: return stream_launch<128, 1, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
-          case 64: return stream_launch<64, 1, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
-          default: break;
-        }
-      } else if (smt == 2) {
-        switch (sbn) {
-          case 256: return stream_launch<256, 2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
-          case 128: return stream_launch<128, 2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
-          case 64: return stream_launch<64, 2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows);
-          default: break;
-        }
-      }
+      if (smt > 0 && (sbn == 128 || sbn == 256))
+        return stream_dispatch<Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows, sbn, smt,
+                                    st.stream_issuers);
     }
     int bn = max_bn;
     const long big_tiles = (long)mt * ((cols + max_bn - 1) / max_bn);

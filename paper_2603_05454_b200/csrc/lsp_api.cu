@@ -619,6 +619,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   else if (key == 17) c->umma.stream_grid_mode = value;
   else if (key == 18) c->umma.stream_even_max_rows = value;
   else if (key == 19) c->umma.stream_two_tiles = value;
+  else if (key == 26) c->umma.stream_issuers = value == 1 ? 1 : 2;
   else if (key == 24) c->umma.stream_big_mt = (value >= 1 && value <= 3) ? value : 0;
   else if (key == 20) c->umma.stream_bn2 = (value == 256 || value == 128 || value == 64) ? value : 0;
   else if (key == 23) c->umma.stream_bn = (value == 256 || value == 128 || value == 64) ? value : 0;
@@ -937,7 +938,7 @@ int lsp_linear_static(const void* A, const void* W, void* out, int M, int N, int
     if (rc == cudaSuccess) rc = cudaDeviceGetAttribute(&sd.max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     if (rc == cudaSuccess) rc = cudaDeviceGetAttribute(&sd.n_sm, cudaDevAttrMultiProcessorCount, dev);
     if (rc == cudaSuccess)
-      rc = cudaFuncSetAttribute(k_gemm_stream<kStaticBN, 1, EpiStore<bf16>>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      rc = cudaFuncSetAttribute(k_gemm_stream<kStaticBN, 1, 2, EpiStore<bf16>>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 sd.max_smem);
     sd.setup_rc = rc;
   });
@@ -976,7 +977,7 @@ int lsp_linear_static(const void* A, const void* W, void* out, int M, int N, int
   }
   StreamArgs args{M, N, n_tiles, 1, 0, kc, a_rows, atoms, kStaticBN / 2, stages, partials, counters, status};
   EpiStore<bf16> epi{(bf16*)out, N};
-  k_gemm_stream<kStaticBN, 1, EpiStore<bf16>><<<grid, UM_THREADS, smem, stream>>>(ma, mb, mb, args, epi);
+  k_gemm_stream<kStaticBN, 1, 2, EpiStore<bf16>><<<grid, ST_THREADS, smem, stream>>>(ma, mb, mb, args, epi);
   e = cudaGetLastError();
   if (e != cudaSuccess) {
     static_msg(err, err_len, "lsp_linear_static: launch failed (%s)", cudaGetErrorString(e));
