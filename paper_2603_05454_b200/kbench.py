@@ -98,14 +98,14 @@ def _fast_weights(sh):
                              w_down=rnd(d, f), attn_norm=one(), ffn_norm=one()) for _ in range(sh.n_layers)])
 
 
-def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False, opts=()):
+def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False, opts=(), batch=0, prompt=0, gen=0):
     """Per-class kernel times of a decode.  layers > 0 cuts the model to its first layers, max_passes > 0 stops each
     decode after that many denoiser passes (both are profiling aids: fewer launches, same kernels and row counts)."""
     wl = S.config(name)
     sh = wl.shape
     if layers > 0:
         sh.n_layers = layers
-    B, P, G = wl.batch, wl.prompt_len, wl.gen_len
+    B, P, G = batch or wl.batch, prompt or wl.prompt_len, gen or wl.gen_len
     w = _fast_weights(sh) if fast_init else S.make_weights(sh, 0, device=DEV)
     dec = LSPDecoder(sh, w, SchedCfg(tau=wl.tau, delim_bitmap=S.delimiter_bitmap(sh.vocab, *wl.delim).to(DEV)), B, P + G,
                      device=DEV)
@@ -148,6 +148,7 @@ def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False, opts=
                 gemm_tflops=round(c["gemm_flops"] / (float(t[1]) * 1e9), 1),
                 attn_gbs=round(c["attn_bytes"] / (float(t[2]) * 1e6), 1),
                 head_gbs=round(c["head_bytes"] / (float(t[3]) * 1e6), 1),
+                attn_tflops=round(c["attn_flops"] / (float(t[2]) * 1e9), 1),
                 append_gbs=round(c["append_bytes"] / max(1e-9, float(t[5]) * 1e6), 1))
 
 
@@ -166,6 +167,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0)
     ap.add_argument("--max-passes", type=int, default=0)
     ap.add_argument("--fast-init", action="store_true")
+    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--prompt", type=int, default=0)
+    ap.add_argument("--gen", type=int, default=0)
     ap.add_argument("--opt", type=int, nargs=2, action="append", default=[], help="lsp_set_option key value")
     a = ap.parse_args()
     if a.what == "gemm":
@@ -175,7 +179,7 @@ def main():
         for m in a.M:
             print(json.dumps(bench_head(m, a.V, a.d, a.reps)), flush=True)
     else:
-        print(json.dumps(bench_decode(a.workload, 1, a.layers, a.max_passes, a.fast_init, a.opt)), flush=True)
+        print(json.dumps(bench_decode(a.workload, 1, a.layers, a.max_passes, a.fast_init, a.opt, a.batch, a.prompt, a.gen)), flush=True)
 
 
 if __name__ == "__main__":
