@@ -135,9 +135,10 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * 22 = fewest two-atom stages the automatic choice accepts, 23 = its tile width for up to 128 rows (0 = automatic,
  * 64, 128 or 256), 24 = row tiles per CTA it uses for more than 256 rows (1, 2,
  * 3 = automatic, default; 0 = the tiled kernel takes those), 25 = launch the step's kernels with programmatic dependent
- * launch, so that each kernel's set-up overlaps its predecessor's tail (1) or plainly (0, default: the step is bound by
- * kernel time, not by launch gaps, and the overlap measured no gain), 26 = MMA-issuing warps of the persistent kernel with one
- * row tile per CTA (1, default, or 2). */
+ * launch (1, default): each kernel's set-up, and a GEMM's first weight tiles, overlap the tail of its predecessor; 0 = plain
+ * launches, 26 = MMA-issuing warps of the persistent kernel with one
+ * row tile per CTA (1, default, or 2), 27 = the persistent kernel caps its shared memory at half an
+ * SM when three pipeline stages still fit, so that its successor can become resident beside it (1, default). */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

@@ -98,6 +98,51 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   auto accf_bar = [&](int b) { return bar_base + 8u * (2 * S + b); };
   auto acce_bar = [&](int b) { return bar_base + 8u * (2 * S + 2 + b); };
 
+  const int G = gridDim.x, g = blockIdx.x;
+  const int RG = args.row_groups;
+  const long T = (long)args.n_tiles * RG;
+  const long U = T * args.kc;
+  // Split shares: CTA g owns the contiguous units [U g / G, U (g + 1) / G).  Whole-tile shares: CTA g owns tiles
+  // g, g + G, g + 2 G, ... (units are then counted within its own tiles), so that the CTAs running at any moment work
+  // on neighbouring tiles: the same few weight tiles for every row group, which keeps the working set inside L2.
+  const long u0 = args.whole_tiles ? 0 : st_first_unit(U, G, g);
+  const long u1 = args.whole_tiles ? ((T - g + G - 1) / G) * args.kc : st_first_unit(U, G, g + 1);
+  const int n_units = (int)(u1 - u0);
+
+  // Position of the producer in the unit space, advanced without divisions (its loop has to keep ahead of the tensor pipe).
+  struct Pos {
+    int vt, c, tile, rg;
+  };
+  auto pos_set = [&](Pos& p, int vt, int c) {
+    p.vt = vt;
+    p.c = c;
+    const int tlin = args.whole_tiles ? g + vt * G : vt;
+    p.tile = tlin / RG;
+    p.rg = tlin % RG;
+  };
+  auto pos_next = [&](Pos& p) {
+    if (++p.c == args.kc) pos_set(p, p.vt + 1, 0);
+  };
+  // weight boxes of one stage: the atoms of a row group back to back (AT x 128 contiguous bytes per weight row)
+  auto load_weights = [&](const Pos& p, int s) {
+    const uint32_t sb = smem_u32(smem + (size_t)s * STAGE_BYTES) + AT * A_ATOM;
+    const int k0 = p.c * AT * UM_BK;
+    for (int b = 0; b < HALF; b += args.box_rows) {
+      int row_b0, row_b1;
+      if (Epi::kDual) { row_b0 = epi.row0(p.tile * HALF + b); row_b1 = epi.row1(p.tile * HALF + b); }
+      else { row_b0 = p.tile * BN + b; row_b1 = p.tile * BN + HALF + b; }
+      for (int j = 0; j < AT; ++j) tma_load_2d(sb + j * B_ATOM + b * 128, &map_b0, k0 + 64 * j, row_b0, full_bar(s));
+      for (int j = 0; j < AT; ++j)
+        tma_load_2d(sb + j * B_ATOM + B_HALF_ATOM + b * 128, &map_b1, k0 + 64 * j, row_b1, full_bar(s));
+    }
+  };
+  auto load_acts = [&](const Pos& p, int s) {
+    const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
+    const int k0 = p.c * AT * UM_BK;
+    for (int j = 0; j < AT; ++j) tma_load_2d(sa + j * A_ATOM, &map_a, k0 + 64 * j, p.rg * ROWS, full_bar(s));
+  };
+
+  const int n_pre = n_units < S ? n_units : S;      // stages whose weights are requested before the predecessor is done
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(full_bar(s), 1);
@@ -111,6 +156,16 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     *epi_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // The weights are never written by any kernel, so the first stages' weight tiles can be requested at once, while a
+    // preceding kernel (launched with programmatic serialisation) is still running; the activations follow after
+    // pdl_wait().  This thread is also the producer below.
+    Pos p;
+    pos_set(p, (int)(u0 / args.kc), (int)(u0 % args.kc));
+    for (int it = 0; it < n_pre; ++it) {
+      mbar_expect_tx(full_bar(it), STAGE_BYTES);
+      load_weights(p, it);
+      pos_next(p);
+    }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -124,55 +179,29 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();          // barriers and tensor memory are set up; from here on the kernel reads what its predecessor wrote
 
-  const int G = gridDim.x, g = blockIdx.x;
-  const int RG = args.row_groups;
-  const long T = (long)args.n_tiles * RG;
-  const long U = T * args.kc;
-  // Split shares: CTA g owns the contiguous units [U g / G, U (g + 1) / G).  Whole-tile shares: CTA g owns tiles
-  // g, g + G, g + 2 G, ... (units are then counted within its own tiles), so that the CTAs running at any moment work
-  // on neighbouring tiles: the same few weight tiles for every row group, which keeps the working set inside L2.
-  const long u0 = args.whole_tiles ? 0 : st_first_unit(U, G, g);
-  const long u1 = args.whole_tiles ? ((T - g + G - 1) / G) * args.kc : st_first_unit(U, G, g + 1);
-
   if (warp == 0) {
     // ---------------- TMA producer: one uninterrupted stream over this CTA's units ----------------
     if (lane == 0) {
       long issued = 0;
-      // position in the unit space, advanced without divisions (this loop has to keep ahead of the tensor pipe)
-      int vt = (int)(u0 / args.kc), c = (int)(u0 % args.kc);
-      int tlin = args.whole_tiles ? g + vt * G : vt;
-      int tile = tlin / RG, rg = tlin % RG;
+      Pos p;
+      pos_set(p, (int)(u0 / args.kc), (int)(u0 % args.kc));
       int s = 0;
       uint32_t ph = 0;
-      const int n_units = (int)(u1 - u0);
       for (int it = 0; it < n_units; ++it) {
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
-          if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 11u; }
-          break;
+        if (it < n_pre) {
+          load_acts(p, s);                   // the stage is armed and its weights are on their way
+        } else {
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
+            if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 11u; }
+            break;
+          }
+          mbar_expect_tx(full_bar(s), STAGE_BYTES);
+          load_weights(p, s);
+          load_acts(p, s);
         }
-        mbar_expect_tx(full_bar(s), STAGE_BYTES);
-        const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
-        const uint32_t sb = sa + AT * A_ATOM;
-        const int k0 = c * AT * UM_BK;
-        // weights first, the atoms of a row group back to back: AT x 128 contiguous bytes per weight row
-        for (int b = 0; b < HALF; b += args.box_rows) {
-          int row_b0, row_b1;
-          if (Epi::kDual) { row_b0 = epi.row0(tile * HALF + b); row_b1 = epi.row1(tile * HALF + b); }
-          else { row_b0 = tile * BN + b; row_b1 = tile * BN + HALF + b; }
-          for (int j = 0; j < AT; ++j) tma_load_2d(sb + j * B_ATOM + b * 128, &map_b0, k0 + 64 * j, row_b0, full_bar(s));
-          for (int j = 0; j < AT; ++j)
-            tma_load_2d(sb + j * B_ATOM + B_HALF_ATOM + b * 128, &map_b1, k0 + 64 * j, row_b1, full_bar(s));
-        }
-        for (int j = 0; j < AT; ++j) tma_load_2d(sa + j * A_ATOM, &map_a, k0 + 64 * j, rg * ROWS, full_bar(s));
         ++issued;
         if (++s == S) { s = 0; ph ^= 1u; }
-        if (++c == args.kc) {
-          c = 0;
-          ++vt;
-          tlin = args.whole_tiles ? g + vt * G : vt;
-          tile = tlin / RG;
-          rg = tlin % RG;
-        }
+        pos_next(p);
       }
       // do not leave while copies may still be landing in this CTA's shared memory
       const long first = issued > S ? issued - S : 0;
@@ -442,7 +471,14 @@ inline StreamShape stream_shape(const UmmaState& st, int a_rows, int bn, int mt,
   sh.atoms = (K % 128 == 0 && (st.max_smem - sh.aux) / (2 * atom) >= st.stream_min_stages2) ? 2 : 1;
   if (st.stream_atoms == 1 || (st.stream_atoms == 2 && K % 128 == 0)) sh.atoms = st.stream_atoms;
   sh.stage_bytes = sh.atoms * atom;
-  sh.stages = (st.max_smem - sh.aux) / sh.stage_bytes;
+  // Half an SM's shared memory when that still gives three stages (it costs no bandwidth, measured): the next kernel's
+  // CTA can then become resident beside this one and request its first weight tiles before this kernel has finished.
+  int budget = st.max_smem;
+  if (st.stream_half_sm) {
+    const int half = (st.sm_smem / 2 - 1024) & ~1023;
+    if (half < budget && (half - sh.aux) / sh.stage_bytes >= 3) budget = half;
+  }
+  sh.stages = (budget - sh.aux) / sh.stage_bytes;
   if (sh.stages > ST_MAX_STAGES) sh.stages = ST_MAX_STAGES;
   if (sh.stages > st.max_stages) sh.stages = st.max_stages;
   return sh;

@@ -481,7 +481,8 @@ struct UmmaState {
   int skinny_ctas_per_sm = 2;      // co-resident CTAs a weight-streaming (M <= 128) launch aims for
   int skinny_min_stages = 3;       // ... provided each still gets this many pipeline stages
   int skinny_bn = 128;             // tile width of plain epilogues in that regime
-  int pdl = 0;                     // launch with the programmatic-serialisation attribute (measured: no gain, off)
+  int pdl = 1;                     // launch with the programmatic-serialisation attribute
+  int stream_half_sm = 1;          // persistent kernel: cap shared memory at half an SM when three stages still fit
   int use_stream = 1;              // M <= 128: use the persistent weight-streaming kernel (gemm_stream.cuh)
   int stream_issuers = 1;          // MMA-issuing warps with one row tile per CTA (two row tiles always use two); measured: no gain from 2
   int stream_two_tiles = 1;        // ... also for 129..256 rows: 1 = two row tiles per CTA, 2 = two row groups, 0 = no

@@ -34,7 +34,7 @@ struct lsp_ctx {
   int max_batch = 0, max_len = 0, max_rows = 0;
   size_t esz = 0;
   cudaStream_t stream = nullptr;
-  int gemm_impl = 1, attn_impl = 1, timing = 0, async_ops = 0, op_repeat = 1, op_rotate = 1, pdl = 0;
+  int gemm_impl = 1, attn_impl = 1, timing = 0, async_ops = 0, op_repeat = 1, op_rotate = 1, pdl = 1;
   // workspace carve (device)
   char *X = nullptr, *Nrm = nullptr, *Qb = nullptr, *Att = nullptr, *Hf = nullptr, *stage = nullptr;
   Top2* part = nullptr;
@@ -619,6 +619,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   else if (key == 17) c->umma.stream_grid_mode = value;
   else if (key == 18) c->umma.stream_even_max_rows = value;
   else if (key == 19) c->umma.stream_two_tiles = value;
+  else if (key == 27) c->umma.stream_half_sm = value ? 1 : 0;
   else if (key == 26) c->umma.stream_issuers = value == 1 ? 1 : 2;
   else if (key == 24) c->umma.stream_big_mt = (value >= 1 && value <= 3) ? value : 0;
   else if (key == 20) c->umma.stream_bn2 = (value == 256 || value == 128 || value == 64) ? value : 0;
