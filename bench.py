@@ -361,6 +361,63 @@ def run_head_bench(dev, peaks, steps, warmup):
                 h2d=host_h.numel() * 2, d2h=B * L * 12, classes=class_report(cnt2, tms, peaks))
 
 
+def run_topology_compare(wl, dev, peaks, warmup):
+    """cfg5: the LSP decode next to the scattered-acceptance baseline (top-k anywhere, k = 32 per step) on the same
+    kernels: denoiser calls, token flips, step latency and KV-append bytes per committed token.  One timed decode per
+    topology; the warm-up decodes use a 64-token generation (they warm the same kernels; a full LSP decode of this
+    workload takes minutes with a random-init model)."""
+    import numpy as np
+    import torch
+    import lsp_synth as S
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+    sh = wl.shape
+    B, P, G = wl.batch, wl.prompt_len, wl.gen_len
+    w = S.make_weights(sh, 0, device=dev)
+    bm = S.delimiter_bitmap(sh.vocab, *wl.delim).to(dev)
+    k = int(wl.extra.get("scattered_k", 32))
+    scheds = {"lsp": SchedCfg(tau=wl.tau, delim_bitmap=bm),
+              "scattered_top_k": SchedCfg(mode=2, fixed_k=k, topology=1)}
+    prompt = S.make_prompt(B, P, sh, 100)
+    tokens = torch.zeros(B, P + G, dtype=torch.int32, device=dev)
+    out = {}
+    dec = LSPDecoder(sh, w, scheds["lsp"], B, P + G, device=dev)
+    for name, sc in scheds.items():
+        dec.set_sched(sc)
+        for _ in range(warmup):
+            tokens[:, :P] = prompt.to(dev)
+            dec.begin(tokens, [P] * B, [64] * B)
+            dec.generate()
+        tokens[:, :P] = prompt.to(dev)
+        dec.reset_counters()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(dev)
+        ev0.record()
+        dec.begin(tokens, [P] * B, [G] * B)
+        n, recs = dec.generate(max_recs=B * (G + 1))
+        ev1.record()
+        torch.cuda.synchronize(dev)
+        ms = ev0.elapsed_time(ev1)
+        assert int((tokens == sh.mask_id).sum()) == 0
+        cnt = dec.counters()
+        # flips between 25 % and 75 % completion of each sequence (the window the paper reports)
+        fl = fb = 0
+        for b in range(B):
+            done = 0
+            for r in recs[b::B]:
+                if r["n_before"] == 0:
+                    continue
+                if 0.25 * G <= done < 0.75 * G:
+                    fl += r["flips"]; fb += r["flip_base"]
+                done += r["L_commit"]
+        out[name] = {"denoiser_calls": n, "tokens_per_s": B * G / (ms * 1e-3), "ms_per_denoiser_step": ms / n,
+                     "decode_ms": ms, "token_flips_25_75": fl, "flip_rate_25_75": (fl / fb) if fb else None,
+                     "kv_append_bytes_per_committed_token": cnt["append_bytes"] / (B * G),
+                     "gpu_launches": int(cnt["launches"]),
+                     "rows_first_last": [sum(r["rows"] for r in recs[:B]), sum(r["rows"] for r in recs[-B:])]}
+    dec.close()
+    return out, k
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -411,6 +468,21 @@ def main():
         return 0
 
     wl = S.config(args.workload)
+    if args.workload == "cfg5":
+        sampler.start()
+        cmp_, k = run_topology_compare(wl, dev, peaks, args.warmup)
+        clocks = sampler.stop()
+        lsp = cmp_["lsp"]
+        line = {"metric": "committed_tokens_per_s", "value": lsp["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1, "steps": 1,
+                "warmup": args.warmup, "ms_per_step": lsp["decode_ms"], "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": f"cfg5: LLaDA-8B shape, batch {wl.batch}, prompt {wl.prompt_len} + {wl.gen_len} masked, "
+                                       f"LSP (tau {wl.tau}) next to scattered top-{k} acceptance, random init",
+                           "warmup_decodes": "64-token generations", "head_scale": wl.shape.head_scale,
+                           "l2": "inputs_exceed_l2"},
+                "topologies": cmp_, "gpu_launches": lsp["gpu_launches"], "clocks": clocks}
+        print(json.dumps(line))
+        return 0
     r = run_decode_bench(wl, dev, rank, world, peaks, args.steps, args.warmup, sampler)
     ms = torch.tensor([r["ms"], r.get("e2e_ms", 0.0)], dtype=torch.float64, device=dev)
     if world > 1:

@@ -72,6 +72,12 @@ typedef struct {
   int exclude_mask_logit;      /* 1: the mask_id column takes no part in argmax / margin / probability */
   float flag_tol;              /* NEAR_THRESHOLD flag: |score_i - tau| <= flag_tol for some i <= L'+1; 0 disables */
   float tie_tol;               /* NEAR_TIE flag: delta_i <= tie_tol for some committed i; 0 disables */
+  int topology;                /* 0 = prefix: commit the left-aligned block yhat_{1:L} (the LSP scheduler);
+                                  1 = scattered acceptance, the baseline the paper compares with (Sec. 4): every pass
+                                  covers the whole generation region and the L most confident masked positions are
+                                  accepted wherever they are (ties: lower position).  L comes from the same policy:
+                                  mode 2 gives top-k with k = fixed_k, modes 0/1 give the "Scattered-Margin" ablation
+                                  (LSP's block sizing, scattered topology).  Only the prompt's K/V are cached. */
 } lsp_sched_cfg;
 
 /* Device pointers to the weights, all element type T.  Per-layer arrays are HOST arrays of
@@ -100,6 +106,8 @@ typedef struct {
   float tau_used;
   unsigned flags;
   float ms;      /* device time of the whole step (same value for every sequence of the batch) */
+  int flips;     /* masked positions whose argmax differs from the previous step's (the paper's token flips, Fig. 3) */
+  int flip_base; /* masked positions that were also scored by the previous step (denominator of the flip rate) */
 } lsp_step_rec;
 
 /* Bytes of workspace lsp_init() needs for up to max_batch sequences of up to max_len positions
@@ -152,7 +160,9 @@ int lsp_begin(lsp_ctx* ctx, int32_t* tokens, int token_stride, const int32_t* pr
  * and changes no committed state.  rec: host [batch] or NULL.  Synchronises the stream. */
 int lsp_denoise_step(lsp_ctx* ctx, lsp_step_rec* rec);
 
-/* Algorithm 1, commit and AppendToCache: writes yhat_{1:L} into the token buffer, appends the pending block's K/V
+/* (Scattered topology: writes the L most confident predictions at their own positions instead, and appends only the
+ * prompt's K/V after the first pass.)
+ * Algorithm 1, commit and AppendToCache: writes yhat_{1:L} into the token buffer, appends the pending block's K/V
  * (computed by the last pass) to the cache as one contiguous copy per layer, and makes the new
  * block pending.  L_override: host [batch] (entries of finished sequences ignored) or NULL to use the
  * proposed lengths.  Needs a preceding lsp_denoise_step; 1 <= L <= N_b else LSP_ERR_STATE and nothing

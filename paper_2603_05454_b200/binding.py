@@ -35,7 +35,7 @@ class ModelCfg(C.Structure):
 class SchedCfgC(C.Structure):
     _fields_ = [("score", C.c_int), ("mode", C.c_int), ("tau", C.c_float), ("alpha", C.c_float), ("beta", C.c_float),
                 ("l_min", C.c_int), ("snap_window", C.c_int), ("fixed_k", C.c_int), ("delim_bitmap", C.c_void_p),
-                ("exclude_mask_logit", C.c_int), ("flag_tol", C.c_float), ("tie_tol", C.c_float)]
+                ("exclude_mask_logit", C.c_int), ("flag_tol", C.c_float), ("tie_tol", C.c_float), ("topology", C.c_int)]
 
 
 class WeightsC(C.Structure):
@@ -45,7 +45,7 @@ class WeightsC(C.Structure):
 
 class StepRec(C.Structure):
     _fields_ = [("step", C.c_int), ("n_before", C.c_int), ("rows", C.c_int), ("l_run", C.c_int), ("l_commit", C.c_int),
-                ("tau_used", C.c_float), ("flags", C.c_uint), ("ms", C.c_float)]
+                ("tau_used", C.c_float), ("flags", C.c_uint), ("ms", C.c_float), ("flips", C.c_int), ("flip_base", C.c_int)]
 
 
 def _load():
@@ -101,11 +101,12 @@ class SchedCfg:
     exclude_mask_logit: int = 1
     flag_tol: float = 0.0
     tie_tol: float = 0.0
+    topology: int = 0         # 0 prefix (LSP), 1 scattered acceptance (baseline)
 
     def to_c(self) -> SchedCfgC:
         p = self.delim_bitmap.data_ptr() if self.delim_bitmap is not None else None
         return SchedCfgC(self.score, self.mode, self.tau, self.alpha, self.beta, self.l_min, self.snap_window,
-                         self.fixed_k, p, self.exclude_mask_logit, self.flag_tol, self.tie_tol)
+                         self.fixed_k, p, self.exclude_mask_logit, self.flag_tol, self.tie_tol, self.topology)
 
 
 def _ptr_array(tensors: Sequence[torch.Tensor]):
@@ -312,4 +313,4 @@ def linear_static(A: torch.Tensor, W: torch.Tensor, out: torch.Tensor, stream=No
 
 def _rec(r: StepRec):
     return dict(step=r.step, n_before=r.n_before, rows=r.rows, L_run=r.l_run, L_commit=r.l_commit,
-                tau_used=r.tau_used, flags=r.flags, ms=r.ms)
+                tau_used=r.tau_used, flags=r.flags, ms=r.ms, flips=r.flips, flip_base=r.flip_base)

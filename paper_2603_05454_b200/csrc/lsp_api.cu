@@ -40,9 +40,10 @@ struct lsp_ctx {
   Top2* part = nullptr;
   int32_t* yhat = nullptr;
   float *pmax = nullptr, *margin = nullptr;
-  int *row_seq = nullptr, *row_pos = nullptr, *head_src = nullptr;
+  int *row_seq = nullptr, *row_pos = nullptr, *head_src = nullptr, *head_pos = nullptr;
+  int32_t* prev_yhat = nullptr;  // [max_batch][max_len] argmax of the previous step per absolute position (-1 = none)
   int* d_desc = nullptr;      // 7 arrays of (max_batch + 1) ints
-  int* d_scan = nullptr;      // 4 arrays of max_batch (run, commit, flags, tau)
+  int* d_scan = nullptr;      // 6 arrays of max_batch (run, commit, flags, tau, flips, flip base)
   float2* rope_cs = nullptr;
   unsigned* d_status = nullptr;
   // pinned host mirrors
@@ -52,7 +53,7 @@ struct lsp_ctx {
   // decode state (host is the authority; the device sees it through the descriptors)
   int32_t* tokens = nullptr;
   int tok_stride = 0, batch = 0, step = 0;
-  std::vector<int> F, Fp, pend, N, Lprop;
+  std::vector<int> F, Fp, pend, N, Lprop, G;
   bool proposed = false;
   int score_rows = 0;
   int last_M = 0;
@@ -151,7 +152,7 @@ struct Carve {
 };
 
 struct Layout {
-  size_t X, Nrm, Qb, Att, Hf, part, yhat, pmax, margin, row_seq, row_pos, head_src, desc, scan, rope, status,
+  size_t X, Nrm, Qb, Att, Hf, part, yhat, pmax, margin, row_seq, row_pos, head_src, head_pos, prev_yhat, desc, scan, rope, status,
       gemm_scratch, gemm_counters, stage, total;
 };
 
@@ -178,8 +179,10 @@ Layout make_layout(const lsp_model_cfg* m, int max_batch, int max_len) {
   L.row_seq = cv.take(R * 4);
   L.row_pos = cv.take(R * 4);
   L.head_src = cv.take(R * 4);
+  L.head_pos = cv.take(R * 4);
+  L.prev_yhat = cv.take(R * 4);
   L.desc = cv.take(7 * (size_t)(max_batch + 1) * 4);
-  L.scan = cv.take(4 * (size_t)max_batch * 4);
+  L.scan = cv.take(6 * (size_t)max_batch * 4);
   L.rope = cv.take((size_t)max_len * (m->head_dim / 2) * sizeof(float2));
   L.status = cv.take(256);
   L.gemm_scratch = cv.take(kGemmScratchBytes);
@@ -261,7 +264,7 @@ ScanParams scan_params(const lsp_ctx* c) {
 }
 
 // merge partials -> scores, scan, copy the scan outputs to the pinned mirror (async)
-int run_merge_scan(lsp_ctx* c, int rows, int n_tiles, const int* d_seq_off, int batch) {
+int run_merge_scan(lsp_ctx* c, int rows, int n_tiles, const int* d_seq_off, int batch, bool count_flips) {
   if (rows > 0) {
     CU(launch_k(c->pdl, k_merge_partials, dim3((rows + 3) / 4), dim3(128), 0, c->stream, (const Top2*)c->part, n_tiles, rows, c->yhat,
                 c->pmax, c->margin));
@@ -269,10 +272,15 @@ int run_merge_scan(lsp_ctx* c, int rows, int n_tiles, const int* d_seq_off, int 
   const float* score = c->s.score == 1 ? c->margin : c->pmax;
   int* o = c->d_scan;
   const int mb = c->max_batch;
+  if (count_flips) {
+    launch_k(c->pdl, k_flip_count, dim3(batch), dim3(256), 0, c->stream, d_seq_off, (const int*)c->head_pos,
+             (const int32_t*)c->yhat, c->prev_yhat, c->max_len, o + 4 * mb, o + 5 * mb);
+    CU(cudaGetLastError());
+  }
   launch_k(c->pdl, k_lsp_scan, dim3(batch), dim3(32), 0, c->stream, score, c->yhat, c->margin, d_seq_off, scan_params(c), o, o + mb,
                                           (uint32_t*)(o + 2 * mb), (float*)(o + 3 * mb));
   CU(cudaGetLastError());
-  CU(cudaMemcpyAsync(c->h_scan, c->d_scan, 4 * (size_t)mb * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaMemcpyAsync(c->h_scan, c->d_scan, 6 * (size_t)mb * 4, cudaMemcpyDeviceToHost, c->stream));
   CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
   return LSP_OK;
 }
@@ -296,12 +304,15 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   const int B = c->batch, s = c->max_batch + 1;
   int* h = c->h_desc;
   int M = 0, Mh = 0, maxQ = 0;
+  const bool scattered = c->s.topology == 1;
   for (int b = 0; b < B; ++b) {
     const int pend = c->N[b] > 0 ? c->pend[b] : 0;
-    const int rows = pend + c->N[b];
+    // rows past the pending block: the masked suffix (prefix topology) or the whole generation region (scattered)
+    const int tail = c->N[b] > 0 ? (scattered ? c->G[b] : c->N[b]) : 0;
+    const int rows = pend + tail;
     h[0 * s + b] = c->F[b];
     h[1 * s + b] = pend;
-    h[2 * s + b] = c->N[b];
+    h[2 * s + b] = tail;
     h[3 * s + b] = M;
     h[4 * s + b] = Mh;
     h[5 * s + b] = c->Fp[b];
@@ -324,10 +335,16 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   T* Hf = (T*)c->Hf;
   seg_begin(c, CLS_MISC);
   launch_k(c->pdl, k_assemble_embed<T>, dim3(M), dim3(128), 0, c->stream, sd, B, c->tokens, c->tok_stride, m.mask_id, (const T*)c->embed, d, X,
-                                               c->row_seq, c->row_pos, c->head_src);
+                                               c->row_seq, c->row_pos, c->head_src, c->head_pos, scattered ? 1 : 0);
+  CU(cudaGetLastError());
+  if (scattered) {
+    launch_k(c->pdl, k_compact_masked, dim3(B), dim3(256), 0, c->stream, sd, (const int32_t*)c->tokens, c->tok_stride, m.mask_id,
+             c->head_src, c->head_pos);
+    CU(cudaGetLastError());
+    count_launch(c, CLS_MISC);
+  }
   seg_end(c);
   count_launch(c, CLS_MISC);
-  CU(cudaGetLastError());
   const size_t plane = (size_t)c->max_rows * kvd;           // elements per staged (layer, K|V) plane
   const size_t cplane = (size_t)c->max_batch * c->max_len * kvd;
   const float scale = 1.0f / sqrtf((float)dh);
@@ -351,7 +368,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
       // algorithmic attention traffic: every key/value row of every sequence once per layer, plus Q and O
       for (int b = 0; b < B; ++b) {
         if (c->N[b] == 0) continue;
-        const double rows_b = c->pend[b] + c->N[b];
+        const double rows_b = c->pend[b] + (scattered ? c->G[b] : c->N[b]);
         c->counters[CNT_ATTN_BYTES] += (2.0 * (c->F[b] + rows_b) * kvd + 2.0 * rows_b * qd) * sizeof(T);
         c->counters[CNT_ATTN_FLOPS] += 4.0 * rows_b * (c->F[b] + rows_b) * qd;
       }
@@ -412,7 +429,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   int rc = run_head<T>(c, Nrm, Mh, &n_tiles);
   if (rc) return rc;
   seg_begin(c, CLS_SCAN);
-  rc = run_merge_scan(c, Mh, n_tiles, sd.head_off, B);
+  rc = run_merge_scan(c, Mh, n_tiles, sd.head_off, B, true);
   seg_end(c);
   count_launch(c, CLS_SCAN, 2);
   c->counters[CNT_STEPS] += 1;
@@ -430,7 +447,9 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
     if (rec) {
       rec[b].step = c->step;
       rec[b].n_before = c->N[b];
-      rec[b].rows = c->N[b] > 0 ? c->pend[b] + c->N[b] : 0;
+      rec[b].rows = c->N[b] > 0 ? c->pend[b] + (scattered ? c->G[b] : c->N[b]) : 0;
+      rec[b].flips = c->N[b] > 0 ? c->h_scan[4 * mb + b] : 0;
+      rec[b].flip_base = c->N[b] > 0 ? c->h_scan[5 * mb + b] : 0;
       rec[b].l_run = c->h_scan[b];
       rec[b].l_commit = c->h_scan[mb + b];
       rec[b].flags = (unsigned)c->h_scan[2 * mb + b];
@@ -551,13 +570,15 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
   c->row_seq = (int*)(ws + L.row_seq);
   c->row_pos = (int*)(ws + L.row_pos);
   c->head_src = (int*)(ws + L.head_src);
+  c->head_pos = (int*)(ws + L.head_pos);
+  c->prev_yhat = (int32_t*)(ws + L.prev_yhat);
   c->d_desc = (int*)(ws + L.desc);
   c->d_scan = (int*)(ws + L.scan);
   c->rope_cs = (float2*)(ws + L.rope);
   c->d_status = (unsigned*)(ws + L.status);
   c->stage = ws + L.stage;
   cudaError_t e = cudaHostAlloc((void**)&c->h_desc, 7 * (size_t)(max_batch + 1) * 4, cudaHostAllocDefault);
-  if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->h_scan, 4 * (size_t)max_batch * 4, cudaHostAllocDefault);
+  if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->h_scan, 6 * (size_t)max_batch * 4, cudaHostAllocDefault);
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->h_status, 16, cudaHostAllocDefault);
   if (e == cudaSuccess) e = cudaEventCreate(&c->ev0);
   if (e == cudaSuccess) e = cudaEventCreate(&c->ev1);
@@ -596,8 +617,11 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
 
 int lsp_set_sched(lsp_ctx* c, const lsp_sched_cfg* sched) {
   if (!c || !sched) return LSP_ERR_ARG;
-  if (sched->mode < 0 || sched->mode > 2 || sched->score < 0 || sched->score > 1)
-    return fail(c, LSP_ERR_ARG, "lsp_set_sched: bad mode/score");
+  if (sched->mode < 0 || sched->mode > 2 || sched->score < 0 || sched->score > 1 || sched->topology < 0 ||
+      sched->topology > 1)
+    return fail(c, LSP_ERR_ARG, "lsp_set_sched: bad mode/score/topology");
+  if (c->tokens && c->step > 0 && sched->topology != c->s.topology)
+    return fail(c, LSP_ERR_STATE, "lsp_set_sched: the topology cannot change in the middle of a decode");
   c->s = *sched;
   return LSP_OK;
 }
@@ -651,7 +675,9 @@ int lsp_begin(lsp_ctx* c, int32_t* tokens, int token_stride, const int32_t* prom
   c->Fp.assign(prompt_len, prompt_len + batch);
   c->pend.assign(prompt_len, prompt_len + batch);   // the prompt is step 0's pending block (CacheInit)
   c->N.assign(gen_len, gen_len + batch);
+  c->G.assign(gen_len, gen_len + batch);
   c->Lprop.assign(batch, 0);
+  CU(cudaMemsetAsync(c->prev_yhat, 0xFF, (size_t)c->max_rows * 4, c->stream));      // -1: no previous prediction
   c->proposed = false;
   // mask fill: reuse the descriptor's F/pend slots to pass P and G
   const int s = c->max_batch + 1;
@@ -697,11 +723,23 @@ int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
   if (chunks > 64) chunks = 64;
   dim3 grid(chunks, m.n_layers * 2, B);
   seg_begin(c, CLS_COMMIT);
-  launch_k(c->pdl, k_commit_append, dim3(grid), dim3(256), 0, c->stream, desc_of(c), (const uint4*)c->stage, (uint4*)c->kv_cache,
-                                               stage_plane_v4, cache_plane_v4, cache_seq_v4, row_v4, c->yhat,
-                                               c->tokens, c->tok_stride);
+  const bool scattered = c->s.topology == 1;
+  if (!scattered || max_pend > 0) {
+    launch_k(c->pdl, k_commit_append, dim3(grid), dim3(256), 0, c->stream, desc_of(c), (const uint4*)c->stage, (uint4*)c->kv_cache,
+                                                 stage_plane_v4, cache_plane_v4, cache_seq_v4, row_v4, c->yhat,
+                                                 c->tokens, c->tok_stride, scattered ? 0 : 1);
+    count_launch(c, CLS_COMMIT);
+  }
+  if (scattered) {
+    // accept the L most confident masked positions wherever they are
+    int max_n = 0;
+    for (int b = 0; b < B; ++b) if (c->N[b] > max_n) max_n = c->N[b];
+    const float* score = c->s.score == 1 ? c->margin : c->pmax;
+    launch_k(c->pdl, k_scatter_commit, dim3(B), dim3(256), (size_t)max_n * sizeof(float), c->stream, desc_of(c), score,
+             (const int32_t*)c->yhat, (const int*)c->head_pos, c->tokens, c->tok_stride);
+    count_launch(c, CLS_COMMIT);
+  }
   seg_end(c);
-  count_launch(c, CLS_COMMIT);
   for (int b = 0; b < B; ++b)
     if (c->N[b] > 0) c->counters[CNT_APPEND_BYTES] += 2.0 * c->pend[b] * kvd * c->esz * 2.0 * m.n_layers;
   CU(cudaGetLastError());
@@ -710,7 +748,7 @@ int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
     c->F[b] += c->pend[b];
     c->counters[CNT_TOKENS] += L[b];
     c->Fp[b] += L[b];
-    c->pend[b] = L[b];
+    c->pend[b] = scattered ? 0 : L[b];       // scattered: nothing becomes pending, the region is recomputed every pass
     c->N[b] -= L[b];
   }
   c->proposed = false;
@@ -792,7 +830,7 @@ int lsp_head_scan(lsp_ctx* c, const void* hidden, const int32_t* seq_offsets, in
                        : run_head<bf16>(c, (const bf16*)hidden, rows, &n_tiles);
   if (rc) return rc;
   seg_begin(c, CLS_SCAN);
-  rc = run_merge_scan(c, rows, n_tiles, c->d_desc + 4 * (c->max_batch + 1), batch);
+  rc = run_merge_scan(c, rows, n_tiles, c->d_desc + 4 * (c->max_batch + 1), batch, false);
   seg_end(c);
   count_launch(c, CLS_SCAN, 2);
   c->counters[CNT_STEPS] += 1;

@@ -13,7 +13,7 @@ template <typename T>
 __global__ void k_assemble_embed(StepDesc sd, int batch, const int32_t* __restrict__ tokens, int tok_stride,
                                  int mask_id, const T* __restrict__ embed, int d, T* __restrict__ X,
                                  int* __restrict__ row_seq, int* __restrict__ row_pos,
-                                 int* __restrict__ head_src) {
+                                 int* __restrict__ head_src, int* __restrict__ head_pos, int scattered) {
   pdl_begin();
   const int r = blockIdx.x;
   int b = 0;
@@ -21,11 +21,16 @@ __global__ void k_assemble_embed(StepDesc sd, int batch, const int32_t* __restri
   const int j = r - sd.row_off[b];
   const int F = sd.F[b], pend = sd.pend[b];
   const int pos = F + j;
-  const int tok = (j < pend) ? tokens[(size_t)b * tok_stride + pos] : mask_id;
+  // prefix topology: rows past the pending block are the masked suffix; scattered topology: every row reads the token
+  // buffer (committed positions hold their token, the others the mask id) and k_compact_masked lists the masked rows
+  const int tok = (scattered || j < pend) ? tokens[(size_t)b * tok_stride + pos] : mask_id;
   if (threadIdx.x == 0) {
     row_seq[r] = b;
     row_pos[r] = pos;
-    if (j >= pend) head_src[sd.head_off[b] + (j - pend)] = r;
+    if (!scattered && j >= pend) {
+      head_src[sd.head_off[b] + (j - pend)] = r;
+      head_pos[sd.head_off[b] + (j - pend)] = pos;
+    }
   }
   const uint4* src = reinterpret_cast<const uint4*>(embed + (size_t)tok * d);
   uint4* dst = reinterpret_cast<uint4*>(X + (size_t)r * d);
@@ -278,7 +283,8 @@ __global__ void k_commit_append(StepDesc sd, const uint4* __restrict__ stage, ui
                                 size_t cache_plane_v4,   // uint4 per (layer, K|V) plane of the cache
                                 size_t cache_seq_v4,     // uint4 per sequence inside a cache plane
                                 int row_v4,              // uint4 per row (n_kv_heads * head_dim * sizeof(T) / 16)
-                                const int32_t* __restrict__ yhat, int32_t* __restrict__ tokens, int tok_stride) {
+                                const int32_t* __restrict__ yhat, int32_t* __restrict__ tokens, int tok_stride,
+                                int write_tokens) {
   pdl_begin();
   const int b = blockIdx.z;
   const int plane = blockIdx.y;
@@ -288,11 +294,108 @@ __global__ void k_commit_append(StepDesc sd, const uint4* __restrict__ stage, ui
   uint4* dst = cache + plane * cache_plane_v4 + b * cache_seq_v4 + (size_t)sd.F[b] * row_v4;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     dst[i] = src[i];
-  if (blockIdx.x == 0 && plane == 0) {
+  if (write_tokens && blockIdx.x == 0 && plane == 0) {
     const int L = sd.Lc[b];
     const int ho = sd.head_off[b];
     int32_t* t = tokens + (size_t)b * tok_stride + sd.Fp[b];
     for (int i = threadIdx.x; i < L; i += blockDim.x) t[i] = yhat[ho + i];
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Scattered topology: lists, in ascending position, the rows of sequence b whose token is still [MASK].
+// One block of 256 threads per sequence; rows [pend_b, pend_b + N_b) of the pass are its generation region.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_compact_masked(StepDesc sd, const int32_t* __restrict__ tokens, int tok_stride,
+                                                        int mask_id, int* __restrict__ head_src,
+                                                        int* __restrict__ head_pos) {
+  __shared__ int warp_cnt[8];
+  __shared__ int base;
+  pdl_begin();
+  const int b = blockIdx.x;
+  const int pend = sd.pend[b], n = sd.N[b], F = sd.F[b], r0 = sd.row_off[b], ho = sd.head_off[b];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  for (int j0 = 0; j0 < n; j0 += 256) {
+    const int j = j0 + threadIdx.x;
+    const int pos = F + pend + j;
+    const bool m = (j < n) && tokens[(size_t)b * tok_stride + pos] == mask_id;
+    const unsigned bal = __ballot_sync(0xffffffffu, m);
+    if (lane == 0) warp_cnt[w] = __popc(bal);
+    __syncthreads();
+    int off = base;
+    for (int i = 0; i < w; ++i) off += warp_cnt[i];
+    if (m) {
+      const int idx = off + __popc(bal & ((1u << lane) - 1u));
+      head_src[ho + idx] = r0 + pend + j;
+      head_pos[ho + idx] = pos;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int t = 0;
+      for (int i = 0; i < 8; ++i) t += warp_cnt[i];
+      base += t;
+    }
+    __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Token flips (Fig. 3): for every masked position of this step, compares its argmax with the one the previous step
+// stored for the same absolute position (-1 = not scored before), counts the differences, and stores the new argmax.
+// One block of 256 threads per sequence.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_flip_count(const int* __restrict__ head_off, const int* __restrict__ head_pos,
+                                                    const int32_t* __restrict__ yhat, int32_t* __restrict__ prev,
+                                                    int prev_stride, int32_t* __restrict__ o_flips,
+                                                    int32_t* __restrict__ o_base) {
+  __shared__ int red[2][8];
+  pdl_begin();
+  const int b = blockIdx.x;
+  const int a = head_off[b], e = head_off[b + 1];
+  int flips = 0, base = 0;
+  for (int i = a + threadIdx.x; i < e; i += 256) {
+    int32_t* p = prev + (size_t)b * prev_stride + head_pos[i];
+    const int32_t old = *p, cur = yhat[i];
+    if (old >= 0) { ++base; flips += (old != cur); }
+    *p = cur;
+  }
+  flips = (int)warp_sum((float)flips);
+  base = (int)warp_sum((float)base);
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = flips; red[1][threadIdx.x >> 5] = base; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int f = 0, t = 0;
+    for (int i = 0; i < 8; ++i) { f += red[0][i]; t += red[1][i]; }
+    o_flips[b] = f;
+    o_base[b] = t;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Scattered commit: accepts the Lc_b most confident masked positions of sequence b (rank by counting: position i
+// is accepted iff fewer than Lc_b positions beat it; a tie goes to the lower position) and writes their predictions
+// into the token buffer at their own positions.  One block of 256 threads per sequence; scores staged in shared
+// memory (dynamic, 4 bytes per masked position of the longest sequence).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_scatter_commit(StepDesc sd, const float* __restrict__ score,
+                                                        const int32_t* __restrict__ yhat, const int* __restrict__ head_pos,
+                                                        int32_t* __restrict__ tokens, int tok_stride) {
+  extern __shared__ float sc_s[];
+  pdl_begin();
+  const int b = blockIdx.x;
+  const int a = sd.head_off[b], n = sd.head_off[b + 1] - a, L = sd.Lc[b];
+  for (int i = threadIdx.x; i < n; i += 256) sc_s[i] = score[a + i];
+  __syncthreads();
+  for (int i = threadIdx.x; i < n; i += 256) {
+    const float si = sc_s[i];
+    int rank = 0;
+    for (int j = 0; j < n; ++j) {
+      const float sj = sc_s[j];
+      rank += (sj > si) || (sj == si && j < i);
+    }
+    if (rank < L) tokens[(size_t)b * tok_stride + head_pos[a + i]] = yhat[a + i];
   }
 }
 
