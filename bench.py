@@ -193,6 +193,21 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------------------
+# replicas: the only cross-rank step is the reduction of the timing
+# ------------------------------------------------------------------------------------------------------------
+def reduce_replicas(ms_local, tokens_local, world, device="cpu"):
+    """Whole-job figures of `world` independent replicas: every rank decodes its own batch, the job takes as long as
+    its slowest rank (MAX over ranks of each entry of ms_local) and commits the sum of the ranks' tokens."""
+    import torch
+    ms = torch.tensor(list(ms_local), dtype=torch.float64, device=device)
+    tok = torch.tensor([float(tokens_local)], dtype=torch.float64, device=device)
+    if world > 1:
+        torch.distributed.all_reduce(ms, op=torch.distributed.ReduceOp.MAX)
+        torch.distributed.all_reduce(tok, op=torch.distributed.ReduceOp.SUM)
+    return [float(x) for x in ms], float(tok[0])
+
+
+# ------------------------------------------------------------------------------------------------------------
 # the CUDA path
 # ------------------------------------------------------------------------------------------------------------
 def class_report(cnt, tms, peaks):
@@ -484,11 +499,7 @@ def main():
         print(json.dumps(line))
         return 0
     r = run_decode_bench(wl, dev, rank, world, peaks, args.steps, args.warmup, sampler)
-    ms = torch.tensor([r["ms"], r.get("e2e_ms", 0.0)], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(ms, op=torch.distributed.ReduceOp.MAX)
-    ms_max, e2e_max = float(ms[0]), float(ms[1])
-    tokens_total = r["tokens"] * world
+    (ms_max, e2e_max), tokens_total = reduce_replicas([r["ms"], r.get("e2e_ms", 0.0)], r["tokens"], world, dev)
     value = tokens_total / (ms_max * 1e-3)
     gemm = r["classes"]["gemm"]
     line = {"metric": "committed_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
