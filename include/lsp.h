@@ -128,7 +128,9 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
 int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
 
 /* Options: key 0 = GEMM implementation for bf16 (0 = CUDA-core reference kernels, 1 = tcgen05,
- * default 1); key 1 = attention implementation for bf16 (0 = CUDA-core, 1 = tensor-core);
+ * default 1); key 1 = attention implementation for bf16 (0 = CUDA-core, 1 = mma.sync tensor cores,
+ * 2 = default: tcgen05 tensor cores for head_dim 128 when a (sequence, KV head) has at least [key 28, default 384] query rows x
+ * group heads, else as 1);
  * key 2 = per-class CUDA-event timing (0 off, 1 on; see lsp_last_timing);
  * key 3 = lsp_op_linear returns without synchronising or checking the device status (1) or not (0);
  * key 4 = lsp_op_linear enqueues the operation this many times (timing aid); key 5 = repetition r reads its weights

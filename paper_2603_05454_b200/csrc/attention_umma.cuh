@@ -1,0 +1,341 @@
+// Suffix-over-prefix attention on the 5th-generation tensor cores (tcgen05 + TMEM), head_dim 128, bf16.
+//
+// Same contract as attention_mma.cuh: the query rows of this pass attend, without any mask, over the contiguous prefix
+// cache [0, F) followed by this pass's staged rows (Sec. 3.2: bidirectional lookahead over the frozen prefix and the
+// active suffix).  One CTA owns 128 "rows" of one (sequence, KV head): a row is a (query position, query head of
+// the group) pair, so grouped-query heads share every K/V tile.
+//
+//   per key tile of 128 keys:   S = Q K^T          tcgen05.mma, A = Q (smem), B = K tile (smem, K-major), D in TMEM
+//                               P = exp2(S - m)    128 threads, one row each: tcgen05.ld, online max / sum, bf16 P to smem
+//                               O += P V           tcgen05.mma, A = P (smem), B = V tile read MN-major (keys are rows)
+//
+// K and V tiles come straight from the cache / staging planes by TMA (two 64-column boxes each, 128-byte swizzle)
+// through a two-stage ring; S is double-buffered in TMEM so that the next tile's QK^T overlaps this tile's softmax.
+// The running maximum is only raised when it grows by more than 8 (log2 units): the accumulator rescale (a TMEM
+// read-modify-write) then happens on the first tiles only, and exp2(S - m) stays below 2^8, which bf16 P and the
+// fp32 row sum hold without loss; the final O / l is the same quantity.
+// Warps 0..3 = softmax + epilogue (warp w owns TMEM lanes 32w..32w+31), warp 4 = TMA producer, warp 5 = TMEM allocator
+// and issuer of the Q K^T MMAs, warp 6 = issuer of the P V MMAs.  Every wait is bounded; on expiry the kernel records (code, site), drains and returns.
+#pragma once
+#include "gemm_umma.cuh"
+
+namespace lsp {
+
+constexpr int AU_BM = 128;        // rows per CTA
+constexpr int AU_BN = 128;        // keys per tile
+constexpr int AU_THREADS = 224;
+constexpr int AU_ATOM = 128 * 128;            // bytes of one [128 rows x 64 bf16] swizzle atom
+constexpr int AU_TILE = 2 * AU_ATOM;          // one 128 x 128 bf16 operand tile
+constexpr int AU_SMEM = 1024 + 2 * AU_TILE /*Q, P*/ + 2 * 2 * AU_TILE /*K, V stages*/ + 256;
+
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const float (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15]))
+      : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane, without waiting: several loads can be in flight before one
+// tc_wait_ld(); the destination must not be read before that wait.
+__device__ __forceinline__ void tc_ld16_nowait(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory descriptor of an MN-major bf16 operand tile stored as [K rows][64 MN elements] atoms with the
+// 128-byte swizzle: 8-row K groups are 1024 bytes apart (stride byte offset), the next 64 MN elements are one atom
+// (16 KB) further (leading byte offset).
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(AU_ATOM >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+// byte offset of 16-byte chunk c (0..15) of row r inside a K-major [128 x 128] bf16 tile made of two swizzled atoms
+__device__ __forceinline__ uint32_t au_swz(int r, int c) {
+  return (uint32_t)((c >> 3) * AU_ATOM + (r >> 3) * 1024 + (r & 7) * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+// grid = (ceil(max rows per sequence * group / 128), n_kv_heads, batch)
+__global__ void __launch_bounds__(AU_THREADS, 1)
+k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ CUtensorMap map_cv,
+            const __grid_constant__ CUtensorMap map_sk, const __grid_constant__ CUtensorMap map_sv,
+            const bf16* __restrict__ q, bf16* __restrict__ out, StepDesc sd, int n_heads, int n_kv_heads, int max_len,
+            float scale_log2, unsigned* status) {
+  constexpr int DH = 128;
+  extern __shared__ uint8_t smem_raw[];
+  pdl_release();
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* Qs = smem;
+  uint8_t* Ps = smem + AU_TILE;
+  uint8_t* KVs = smem + 2 * AU_TILE;                    // stage s: K at s * 2 * AU_TILE, V right behind it
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 6 * AU_TILE);
+  // bars: 0,1 kv_full; 2,3 kv_empty; 4,5 s_full; 6,7 s_empty; 8 p_ready; 9 pv_done
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  const uint32_t bb = smem_u32(bars);
+  auto bar = [&](int i) { return bb + 8u * i; };
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  const int b = blockIdx.z, kvh = blockIdx.y;
+  const int G = n_heads / n_kv_heads;
+  if (threadIdx.x == 0) {
+    mbar_init(bar(0), 1); mbar_init(bar(1), 1);
+    mbar_init(bar(2), 1); mbar_init(bar(3), 1);
+    mbar_init(bar(4), 1); mbar_init(bar(5), 1);
+    mbar_init(bar(6), 4); mbar_init(bar(7), 4);
+    mbar_init(bar(8), 4);
+    mbar_init(bar(9), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+
+  const int r0 = sd.row_off[b];
+  const int Qn = sd.row_off[b + 1] - r0;
+  const int rows_total = Qn * G;
+  const int row_base = blockIdx.x * AU_BM;
+  const int F = sd.F[b];
+  const int n_c = (F + AU_BN - 1) / AU_BN, n_s = (Qn + AU_BN - 1) / AU_BN;
+  const int n_tiles = (row_base < rows_total) ? n_c + n_s : 0;     // a CTA past the last row does nothing
+  const int ldq = n_heads * DH;
+
+  if (warp < 4) {
+    // ---- Q tile -> swizzled shared memory (zeros for rows past the end)
+    const int r = threadIdx.x;
+    const int row = row_base + r;
+    const bool valid = row < rows_total;
+    if (n_tiles > 0) {
+      const int qi = valid ? row / G : 0, hg = valid ? row % G : 0;
+      const uint4* src = reinterpret_cast<const uint4*>(q + (size_t)(r0 + qi) * ldq + (kvh * G + hg) * DH);
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const uint4 v = valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(Qs + au_swz(r, c)) = v;
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+  }
+  __syncthreads();      // Q is in place
+
+  if (warp == 4) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      for (int t = 0; t < n_tiles; ++t) {
+        const int s = t & 1;
+        if (!mbar_wait(bar(2 + s), ((uint32_t)(t >> 1) & 1u) ^ 1u, abort_flag)) {
+          if (!*abort_flag) { *abort_flag = 1; atomicExch(status, 1u); status[1] = 21u; }
+          break;
+        }
+        mbar_expect_tx(bar(s), 2 * AU_TILE);
+        const uint32_t kd = smem_u32(KVs + (size_t)s * 2 * AU_TILE), vd = kd + AU_TILE;
+        const bool cache = t < n_c;
+        const int row = cache ? b * max_len + t * AU_BN : r0 + (t - n_c) * AU_BN;
+        const CUtensorMap* mk = cache ? &map_ck : &map_sk;
+        const CUtensorMap* mv = cache ? &map_cv : &map_sv;
+        tma_load_2d(kd, mk, kvh * DH, row, bar(s));
+        tma_load_2d(kd + AU_ATOM, mk, kvh * DH + 64, row, bar(s));
+        tma_load_2d(vd, mv, kvh * DH, row, bar(s));
+        tma_load_2d(vd + AU_ATOM, mv, kvh * DH + 64, row, bar(s));
+        ++issued;
+      }
+      for (int t = issued > 2 ? issued - 2 : 0; t < issued; ++t) {
+        volatile uint32_t no_abort = 0;
+        mbar_wait(bar(t & 1), (uint32_t)(t >> 1) & 1u, &no_abort);
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------- MMA issuer 1: S = Q K^T of every tile ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = make_idesc(AU_BN);
+      for (int t = 0; t < n_tiles; ++t) {
+        const int s = t & 1;
+        if (!mbar_wait(bar(s), (uint32_t)(t >> 1) & 1u, abort_flag) ||
+            !mbar_wait(bar(6 + s), ((uint32_t)(t >> 1) & 1u) ^ 1u, abort_flag)) {
+          if (!*abort_flag) { *abort_flag = 1; atomicExch(status, 1u); status[1] = 22u; }
+          break;
+        }
+        tc_fence_after();
+        const uint32_t kd = smem_u32(KVs + (size_t)s * 2 * AU_TILE);
+        const uint32_t d = tmem_base + 128u + (uint32_t)(s * AU_BN);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint64_t da = make_smem_desc(smem_u32(Qs) + (k >> 2) * AU_ATOM) + (uint64_t)(2 * (k & 3));
+          const uint64_t db = make_smem_desc(kd + (k >> 2) * AU_ATOM) + (uint64_t)(2 * (k & 3));
+          tc_mma_f16(d, da, db, idesc_qk, k ? 1u : 0u);
+        }
+        tc_commit(bar(4 + s));
+      }
+    }
+  } else if (warp == 6) {
+    // ---------------- MMA issuer 2: O += P V of every tile (a second issuing warp doubles the issue rate) ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_pv = make_idesc(DH) | (1u << 16);          // B operand (V) is MN-major
+      for (int t = 0; t < n_tiles; ++t) {
+        const int s = t & 1;
+        if (!mbar_wait(bar(s), (uint32_t)(t >> 1) & 1u, abort_flag) || !mbar_wait(bar(8), (uint32_t)t & 1u, abort_flag)) {
+          if (!*abort_flag) { *abort_flag = 1; atomicExch(status, 1u); status[1] = 23u; }
+          break;
+        }
+        tc_fence_after();
+        const uint32_t vd = smem_u32(KVs + (size_t)s * 2 * AU_TILE) + AU_TILE;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {          // 16 keys per step
+          const uint64_t da = make_smem_desc(smem_u32(Ps) + (k >> 2) * AU_ATOM) + (uint64_t)(2 * (k & 3));
+          const uint64_t db = make_smem_desc_mn(vd) + (uint64_t)(k * (2048 >> 4));
+          tc_mma_f16(tmem_base, da, db, idesc_pv, (t | k) ? 1u : 0u);
+        }
+        tc_commit(bar(2 + s));      // K/V stage free (its Q K^T finished before this tile's softmax began)
+        tc_commit(bar(9));          // P free, O updated
+      }
+    }
+  } else {
+    // ---------------- softmax + epilogue (warps 0..3, one row per thread) ----------------
+    const int r = threadIdx.x;
+    const uint32_t lane_base = tmem_base + ((uint32_t)(warp * 32) << 16);
+    float m_used = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int t = 0; t < n_tiles; ++t) {
+      const int s = t & 1;
+      if (!mbar_wait(bar(4 + s), (uint32_t)(t >> 1) & 1u, abort_flag)) {
+        if (lane == 0 && !*abort_flag) { *abort_flag = 1; atomicExch(status, 1u); status[1] = 24u; }
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const int valid_keys = (t < n_c) ? min(AU_BN, F - t * AU_BN) : min(AU_BN, Qn - (t - n_c) * AU_BN);
+      float sv[AU_BN];
+#pragma unroll
+      for (int c = 0; c < AU_BN; c += 16) tc_ld16_nowait(lane_base + 128u + (uint32_t)(s * AU_BN + c), sv + c);
+      tc_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(6 + s));          // S buffer read
+      // raw scores; the scale (positive) is folded into the exponent's FMA, masking only touches a ragged last tile
+      if (valid_keys < AU_BN) {
+#pragma unroll
+        for (int i = 0; i < AU_BN; ++i)
+          if (i >= valid_keys) sv[i] = -INFINITY;
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < AU_BN; ++i) mx = fmaxf(mx, sv[i]);
+      mx *= scale_log2;
+      float corr = 1.f;
+      bool raise = false;
+      if (mx > m_used + 8.f) {                          // also the first tile (m_used = -inf)
+        corr = ex2_approx(m_used - mx);                 // 0 on the first tile
+        m_used = mx;
+        raise = t > 0;
+      }
+      float sum = 0.f;
+      uint32_t pk[AU_BN / 2];
+      const float neg_m = -m_used;
+#pragma unroll
+      for (int i = 0; i < AU_BN; i += 2) {
+        const float p0 = ex2_approx(fmaf(sv[i], scale_log2, neg_m)), p1 = ex2_approx(fmaf(sv[i + 1], scale_log2, neg_m));
+        sum += p0 + p1;
+        const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+        pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+      }
+      l = l * corr + sum;
+      if (t > 0) {
+        // P and O are free once the previous tile's P V has completed
+        if (!mbar_wait(bar(9), (uint32_t)(t - 1) & 1u, abort_flag)) {
+          if (lane == 0 && !*abort_flag) { *abort_flag = 1; atomicExch(status, 1u); status[1] = 25u; }
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, raise)) {           // rare after the first tiles: rescale the accumulator rows
+#pragma unroll 1
+          for (int c = 0; c < DH; c += 16) {
+            float v[16];
+            tc_ld16(lane_base + (uint32_t)c, v);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] *= corr;
+            tc_st16(lane_base + (uint32_t)c, v);
+          }
+          tc_wait_st();
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < 16; ++c)
+        *reinterpret_cast<uint4*>(Ps + au_swz(r, c)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(8));               // P ready
+    }
+    if (ok && n_tiles > 0 && mbar_wait(bar(9), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
+      tc_fence_after();
+      const int row = row_base + r;
+      const float inv = 1.f / l;
+      const bool valid = row < rows_total;
+      const int qi = valid ? row / G : 0, hg = valid ? row % G : 0;
+      uint4* dst = reinterpret_cast<uint4*>(out + (size_t)(r0 + qi) * ldq + (kvh * G + hg) * DH);
+#pragma unroll 1
+      for (int c = 0; c < DH; c += 16) {
+        float v[16];
+        tc_ld16(lane_base + (uint32_t)c, v);
+        if (valid) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] *= inv;
+          dst[c >> 3] = pack8(v);
+          dst[(c >> 3) + 1] = pack8(v + 8);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// 2-D bf16 tensor map of a K or V plane [rows, kvd] with a box of 64 columns x 128 rows (one swizzle atom).
+inline bool attn_umma_map(UmmaState& st, CUtensorMap* m, const void* base, size_t rows, int kvd) {
+  cuuint64_t dims[2] = {(cuuint64_t)kvd, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)kvd * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)AU_BN};
+  cuuint32_t estr[2] = {1, 1};
+  return st.encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace lsp

@@ -17,6 +17,7 @@
 #include "misc_kernels.cuh"
 #ifndef LSP_NO_UMMA
 #include "gemm_stream.cuh"
+#include "attention_umma.cuh"
 #endif
 
 using namespace lsp;
@@ -34,7 +35,7 @@ struct lsp_ctx {
   int max_batch = 0, max_len = 0, max_rows = 0;
   size_t esz = 0;
   cudaStream_t stream = nullptr;
-  int gemm_impl = 1, attn_impl = 1, timing = 0, async_ops = 0, op_repeat = 1, op_rotate = 1, pdl = 1;
+  int gemm_impl = 1, attn_impl = 2, timing = 0, async_ops = 0, op_repeat = 1, op_rotate = 1, pdl = 1, attn_umma_min_rows = 384;
   // workspace carve (device)
   char *X = nullptr, *Nrm = nullptr, *Qb = nullptr, *Att = nullptr, *Hf = nullptr, *stage = nullptr;
   Top2* part = nullptr;
@@ -66,6 +67,7 @@ struct lsp_ctx {
   std::string err;
 #ifndef LSP_NO_UMMA
   UmmaState umma;
+  std::vector<CUtensorMap> attn_maps;    // per layer: cache K, cache V, staging K, staging V (tcgen05 attention)
 #endif
 };
 
@@ -375,8 +377,23 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
       count_launch(c, CLS_ATTN);
       seg_begin(c, CLS_ATTN);
       bool done = false;
+#ifndef LSP_NO_UMMA
       if constexpr (std::is_same<T, bf16>::value) {
-        if (c->attn_impl == 1) {
+        // the tcgen05 kernel works on 128-row tiles: it pays from a few tiles per (sequence, KV head) upwards; below that
+        // the 64-row mma.sync kernel has more CTAs in flight
+        if (c->attn_impl == 2 && dh == 128 && !c->attn_maps.empty() && maxQ * (m.n_heads / m.n_kv_heads) >= c->attn_umma_min_rows) {
+          const int G = m.n_heads / m.n_kv_heads;
+          dim3 g3((maxQ * G + AU_BM - 1) / AU_BM, m.n_kv_heads, B);
+          const float sl2 = scale * 1.4426950408889634f;
+          const CUtensorMap* mp = &c->attn_maps[4 * l];
+          launch_k(c->pdl, k_attn_umma, g3, dim3(AU_THREADS), (size_t)AU_SMEM, c->stream, mp[0], mp[1], mp[2], mp[3],
+                   (const bf16*)Qb, Att, sd, m.n_heads, m.n_kv_heads, c->max_len, sl2, c->d_status);
+          done = true;
+        }
+      }
+#endif
+      if constexpr (std::is_same<T, bf16>::value) {
+        if (!done && c->attn_impl >= 1) {
           const int G = m.n_heads / m.n_kv_heads;
           dim3 g2((maxQ * G + AM_BM - 1) / AM_BM, m.n_kv_heads, B);
           const float sl2 = scale * 1.4426950408889634f;
@@ -609,6 +626,22 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
       lsp_destroy(c);
       return LSP_ERR_CUDA;
     }
+    if (model->head_dim == 128) {
+      // tensor maps of the K / V planes for the tcgen05 attention kernel
+      const int kvd = model->n_kv_heads * model->head_dim;
+      const size_t plane = (size_t)max_batch * max_len * kvd * 2;      // bytes of one (layer, K|V) plane, cache and staging alike
+      c->attn_maps.resize((size_t)4 * model->n_layers);
+      bool ok = cudaFuncSetAttribute(k_attn_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, AU_SMEM) == cudaSuccess;
+      for (int l = 0; l < model->n_layers && ok; ++l) {
+        const char* ck = c->kv_cache + (size_t)(2 * l) * plane;
+        const char* sk = c->stage + (size_t)(2 * l) * plane;
+        ok = attn_umma_map(c->umma, &c->attn_maps[4 * l + 0], ck, (size_t)max_batch * max_len, kvd) &&
+             attn_umma_map(c->umma, &c->attn_maps[4 * l + 1], ck + plane, (size_t)max_batch * max_len, kvd) &&
+             attn_umma_map(c->umma, &c->attn_maps[4 * l + 2], sk, (size_t)max_batch * max_len, kvd) &&
+             attn_umma_map(c->umma, &c->attn_maps[4 * l + 3], sk + plane, (size_t)max_batch * max_len, kvd);
+      }
+      if (!ok) c->attn_maps.clear();      // the mma.sync kernel takes over
+    }
   }
 #endif
   *out = c;
@@ -620,8 +653,11 @@ int lsp_set_sched(lsp_ctx* c, const lsp_sched_cfg* sched) {
   if (sched->mode < 0 || sched->mode > 2 || sched->score < 0 || sched->score > 1 || sched->topology < 0 ||
       sched->topology > 1)
     return fail(c, LSP_ERR_ARG, "lsp_set_sched: bad mode/score/topology");
-  if (c->tokens && c->step > 0 && sched->topology != c->s.topology)
-    return fail(c, LSP_ERR_STATE, "lsp_set_sched: the topology cannot change in the middle of a decode");
+  if (sched->topology != c->s.topology && c->tokens && c->step > 0) {
+    bool active = false;
+    for (int b = 0; b < c->batch; ++b) active |= c->N[b] > 0;
+    if (active) return fail(c, LSP_ERR_STATE, "lsp_set_sched: the topology cannot change in the middle of a decode");
+  }
   c->s = *sched;
   return LSP_OK;
 }
@@ -630,6 +666,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   if (!c) return LSP_ERR_ARG;
   if (key == 0) c->gemm_impl = value;
   else if (key == 1) c->attn_impl = value;
+  else if (key == 28) c->attn_umma_min_rows = value;
   else if (key == 2) c->timing = value;
   else if (key == 3) c->async_ops = value;
   else if (key == 4) c->op_repeat = value < 1 ? 1 : value;

@@ -169,3 +169,13 @@ def test_state_errors_leave_state_unchanged():
     with pytest.raises(LSPError):
         dec.denoise_step()                      # already finished
     dec.close()
+
+
+@pytest.mark.parametrize("hq,hkv", [(4, 4), (4, 2), (7, 1)])
+def test_bf16_tcgen05_attention_head_dim_128(hq, hkv):
+    """The tcgen05/TMEM attention kernel (option key 1 = 2): MHA and grouped-query packing, several key tiles from the
+    cache and from the staged rows, ragged tails on both."""
+    from paper_2603_05454_b200 import SchedCfg
+    sh = S.ModelShape(2, 128 * hq, hq, hkv, 128, 512, 2048, dtype="bf16", head_scale=1.5, w_std=0.5 / (128 * hq) ** 0.5)
+    _teacher_forced(sh, 11, 150, 170, SchedCfg(mode=2, fixed_k=45), (1, 200), attn_impl=2, max_steps=4)
+    _teacher_forced(sh, 12, 40, 90, SchedCfg(tau=0.04), (1, 400), attn_impl=2, max_steps=6)
