@@ -148,7 +148,9 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * launch (1, default): each kernel's set-up, and a GEMM's first weight tiles, overlap the tail of its predecessor; 0 = plain
  * launches, 26 = MMA-issuing warps of the persistent kernel with one
  * row tile per CTA (1, default, or 2), 27 = the persistent kernel caps its shared memory at half an
- * SM when three pipeline stages still fit, so that its successor can become resident beside it (1, default). */
+ * SM when three pipeline stages still fit, so that its successor can become resident beside it (1, default),
+ * 28 = see key 1, 29 = the K slices of a split tile run as one thread block cluster and are reduced through distributed
+ * shared memory (1, default) or through global scratch by the last CTA to arrive (0). */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

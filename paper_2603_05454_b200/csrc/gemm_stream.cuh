@@ -38,6 +38,8 @@ struct StreamArgs {
   int row_groups;   // groups of 128 MT activation rows (1 when M <= 128 MT); a tile is (column tile, row group), row
                     // group fastest, so a CTA meets the same weight tile again while it is still in L2
   int whole_tiles;  // 1: shares are whole tiles (no tile is split between CTAs)
+  int cluster;      // > 1: the launch uses thread block clusters of this size, one cluster per tile, CTA rank r owning the
+                    // r-th K slice; the partial tiles are then reduced through distributed shared memory (see the kernel)
   int kc;           // K chunks (one per stage) per tile
   int a_rows;       // activation box rows (M rounded up to a multiple of 8)
   int atoms;        // 64-element K atoms per stage (1 or 2)
@@ -50,6 +52,27 @@ struct StreamArgs {
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// thread block cluster helpers
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ unsigned cluster_ctarank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address, in the cluster's shared window, of this CTA's shared address saddr as seen in CTA `rank`
+__device__ __forceinline__ uint32_t cluster_map(uint32_t saddr, unsigned rank) {
+  uint32_t d;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(d) : "r"(saddr), "r"(rank));
+  return d;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
 }
 
 // first unit of CTA g when U units are dealt to G CTAs
@@ -108,6 +131,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   const long u0 = args.whole_tiles ? 0 : st_first_unit(U, G, g);
   const long u1 = args.whole_tiles ? ((T - g + G - 1) / G) * args.kc : st_first_unit(U, G, g + 1);
   const int n_units = (int)(u1 - u0);
+  int cl_tile = 0, cl_row0 = 0;      // cluster mode: the tile this CTA contributed a K slice to
 
   // Position of the producer in the unit space, advanced without divisions (its loop has to keep ahead of the tensor pipe).
   struct Pos {
@@ -326,7 +350,11 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         // publish this CTA's partial tile, then count its chunks in; the CTA that completes the count finishes the tile.
         // Partial tile layout: [16-column chunk][quarter][row][4 floats], so that the lanes of a warp (consecutive
         // rows) write and read consecutive 16-byte pieces.
-        float4* slot_base = reinterpret_cast<float4*>(args.scratch + (size_t)(g * 2 + (seg == 0 ? 0 : 1)) * ROWS * BN);
+        // With clusters the partial tile goes to this CTA's own shared memory (the pipeline stages are idle by now) and
+        // is reduced after the role loops; without, to the global scratch slot of this CTA.
+        float4* slot_base = args.cluster > 1
+                                ? reinterpret_cast<float4*>(smem)
+                                : reinterpret_cast<float4*>(args.scratch + (size_t)(g * 2 + (seg == 0 ? 0 : 1)) * ROWS * BN);
 #pragma unroll 1
         for (int mt = 0; mt < MT; ++mt) {
           const int m = mt * UM_BM + r_in;              // row within the row group
@@ -351,6 +379,12 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(acce_bar(buf));
+        if (args.cluster > 1) {          // reduced after the cluster barrier below
+          cl_tile = tile;
+          cl_row0 = row0;
+          u = seg_end;
+          continue;
+        }
         __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (threadIdx.x == 64) {
@@ -435,6 +469,53 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
       u = seg_end;
     }
   }
+  if (args.cluster > 1) {
+    // Split-K reduction inside the cluster: every CTA's partial tile sits in its shared memory; after the barrier CTA
+    // rank r sums, for its share of the 16-column chunks, the partials of all ranks in rank order (= K order, so the
+    // result does not depend on timing) straight from their shared memory, and runs the fused epilogue on them.
+    // Every thread of every CTA reaches both barriers (no early exits above), so they cannot hang.
+    const int C = args.cluster;
+    cluster_sync();
+    if constexpr (!Epi::kReduce) {
+      if (warp >= 2 && warp <= 5 && n_units > 0) {
+        constexpr int CH = Epi::kDual ? HALF : BN;
+        constexpr int NCH = CH / 16;
+        const unsigned rank = cluster_ctarank();
+        const int ch_lo = NCH * (int)rank / C, ch_hi = NCH * ((int)rank + 1) / C;
+        const int rows_here = min(ROWS, args.M - cl_row0);
+        const int n_items = rows_here * (ch_hi - ch_lo);
+        const uint32_t base = smem_u32(smem);
+        for (int idx = threadIdx.x - 64; idx < n_items; idx += 128) {
+          const int mm = idx % rows_here, ch = ch_lo + idx / rows_here, c = ch * 16;
+          float a0[16], a1[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
+          const uint32_t off0 = (uint32_t)(((c >> 4) * 4 * ROWS + mm) * 16);
+          const uint32_t off1 = (uint32_t)((((HALF + c) >> 4) * 4 * ROWS + mm) * 16);
+          for (int pr = 0; pr < C; ++pr) {
+            const uint32_t peer = cluster_map(base, (unsigned)pr);
+            float4 t0[4], t1[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) t0[i] = ld_cluster_f4(peer + off0 + (uint32_t)(i * ROWS * 16));
+            if (Epi::kDual) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) t1[i] = ld_cluster_f4(peer + off1 + (uint32_t)(i * ROWS * 16));
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              a0[4 * i] += t0[i].x; a0[4 * i + 1] += t0[i].y; a0[4 * i + 2] += t0[i].z; a0[4 * i + 3] += t0[i].w;
+              if (Epi::kDual) {
+                a1[4 * i] += t1[i].x; a1[4 * i + 1] += t1[i].y; a1[4 * i + 2] += t1[i].z; a1[4 * i + 3] += t1[i].w;
+              }
+            }
+          }
+          const int j0 = cl_tile * CH;
+          if (j0 + c < args.n_pairs) epi16(epi, cl_row0 + mm, j0 + c, a0, a1);
+        }
+      }
+    }
+    cluster_sync();      // nobody leaves while a peer may still read its shared memory
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -513,9 +594,19 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
   const int whole = (row_groups > 1 && T >= st.n_sm) ? 1 : 0;
   int grid = whole ? st.n_sm : stream_grid(st, (int)T, M);
   if (grid > T * kc) grid = (int)(T * kc);
-  StreamArgs args{M, NP, n_tiles, row_groups, whole, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch, st.counters,
-                  status};
-  cudaError_t e = launch_k(st.pdl, k_gemm_stream<BN, MT, NI, Epi>, dim3(grid), dim3(ST_THREADS), smem, stream, *ma, *mb0, *mb1, args, epi);
+  // K slices of one tile on the CTAs of one cluster: the reduction then stays on chip
+  int cluster = 0;
+  if (!whole && !Epi::kReduce && st.stream_cluster && grid % T == 0) {
+    const int splits = (int)(grid / T);
+    // sizes 2, 4 and 8 only: a cluster of 3 measured 40 % slower than the same split without clusters
+    if ((splits == 2 || splits == 4 || splits == 8) && kc >= splits &&
+        (size_t)sh.stages * sh.stage_bytes >= (size_t)UM_BM * MT * BN * sizeof(float))
+      cluster = splits;
+  }
+  StreamArgs args{M, NP, n_tiles, row_groups, whole, cluster, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch,
+                  st.counters, status};
+  cudaError_t e = launch_k(st.pdl, k_gemm_stream<BN, MT, NI, Epi>, dim3(grid), dim3(ST_THREADS), smem, stream, cluster, *ma, *mb0,
+                           *mb1, args, epi);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
   return 0;

@@ -681,6 +681,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   else if (key == 18) c->umma.stream_even_max_rows = value;
   else if (key == 19) c->umma.stream_two_tiles = value;
   else if (key == 27) c->umma.stream_half_sm = value ? 1 : 0;
+  else if (key == 29) c->umma.stream_cluster = value ? 1 : 0;
   else if (key == 26) c->umma.stream_issuers = value == 1 ? 1 : 2;
   else if (key == 24) c->umma.stream_big_mt = (value >= 1 && value <= 3) ? value : 0;
   else if (key == 20) c->umma.stream_bn2 = (value == 256 || value == 128 || value == 64) ? value : 0;
@@ -1051,7 +1052,7 @@ int lsp_linear_static(const void* A, const void* W, void* out, int M, int N, int
     static_msg(err, err_len, "lsp_linear_static: clearing the counters failed (%s)", cudaGetErrorString(e));
     return LSP_ERR_CUDA;
   }
-  StreamArgs args{M, N, n_tiles, 1, 0, kc, a_rows, atoms, kStaticBN / 2, stages, partials, counters, status};
+  StreamArgs args{M, N, n_tiles, 1, 0, 0, kc, a_rows, atoms, kStaticBN / 2, stages, partials, counters, status};
   EpiStore<bf16> epi{(bf16*)out, N};
   k_gemm_stream<kStaticBN, 1, 2, EpiStore<bf16>><<<grid, ST_THREADS, smem, stream>>>(ma, mb, mb, args, epi);
   e = cudaGetLastError();
