@@ -535,7 +535,13 @@ inline size_t stream_scratch_bytes(int n_ctas, int bn, int mt) { return (size_t)
 // the second choice is as fast or faster at every row count from 2 to 128, so it is the default.
 inline int stream_grid(const UmmaState& st, int n_tiles, int M) {
   if (st.target_ctas > 0) return st.target_ctas;
-  const int aligned = n_tiles <= st.n_sm ? n_tiles * (st.n_sm / n_tiles) : st.n_sm;
+  int splits = n_tiles <= st.n_sm ? st.n_sm / n_tiles : 0;
+  if (st.stream_cluster && splits > 1) {          // a split of 2, 4 or 8 can run as a thread block cluster
+    int p2 = 1;
+    while (2 * p2 <= splits && 2 * p2 <= 8) p2 *= 2;
+    splits = p2;
+  }
+  const int aligned = splits > 0 ? n_tiles * splits : st.n_sm;
   if (st.stream_grid_mode == 1) return st.n_sm;
   if (st.stream_grid_mode == 2) return aligned;
   return M <= st.stream_even_max_rows ? st.n_sm : aligned;
