@@ -129,7 +129,7 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
 
 /* Options: key 0 = GEMM implementation for bf16 (0 = CUDA-core reference kernels, 1 = tcgen05,
  * default 1); key 1 = attention implementation for bf16 (0 = CUDA-core, 1 = mma.sync tensor cores,
- * 2 = default: tcgen05 tensor cores for head_dim 128 when a (sequence, KV head) has at least [key 28, default 384] query rows x
+ * 2 = default: tcgen05 tensor cores for head_dim 128 when a (sequence, KV head) has at least [key 28, default 0] query rows x
  * group heads, else as 1);
  * key 2 = per-class CUDA-event timing (0 off, 1 on; see lsp_last_timing);
  * key 3 = lsp_op_linear returns without synchronising or checking the device status (1) or not (0);
@@ -149,7 +149,8 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * launches, 26 = MMA-issuing warps of the persistent kernel with one
  * row tile per CTA (1, default, or 2), 27 = the persistent kernel caps its shared memory at half an
  * SM when three pipeline stages still fit, so that its successor can become resident beside it (1, default),
- * 28 = see key 1, 29 = the K slices of a split tile run as one thread block cluster and are reduced through distributed
+ * 28 = see key 1, 30 = the tcgen05 attention splits a row tile's keys over a thread block cluster when there are few CTAs
+ * (1, default), 29 = the K slices of a split tile run as one thread block cluster and are reduced through distributed
  * shared memory (1, default) or through global scratch by the last CTA to arrive (0). */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 

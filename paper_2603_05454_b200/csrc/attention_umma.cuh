@@ -17,7 +17,7 @@
 // Warps 0..3 = softmax + epilogue (warp w owns TMEM lanes 32w..32w+31), warp 4 = TMA producer, warp 5 = TMEM allocator
 // and issuer of the Q K^T MMAs, warp 6 = issuer of the P V MMAs.  Every wait is bounded; on expiry the kernel records (code, site), drains and returns.
 #pragma once
-#include "gemm_umma.cuh"
+#include "gemm_stream.cuh"
 
 namespace lsp {
 
@@ -57,6 +57,11 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float ld_cluster_f1(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory descriptor of an MN-major bf16 operand tile stored as [K rows][64 MN elements] atoms with the
@@ -82,7 +87,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1)
 k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ CUtensorMap map_cv,
             const __grid_constant__ CUtensorMap map_sk, const __grid_constant__ CUtensorMap map_sv,
             const bf16* __restrict__ q, bf16* __restrict__ out, StepDesc sd, int n_heads, int n_kv_heads, int max_len,
-            float scale_log2, unsigned* status) {
+            float scale_log2, int cluster, unsigned* status) {
   constexpr int DH = 128;
   extern __shared__ uint8_t smem_raw[];
   pdl_release();
@@ -125,10 +130,15 @@ k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ 
   const int r0 = sd.row_off[b];
   const int Qn = sd.row_off[b + 1] - r0;
   const int rows_total = Qn * G;
-  const int row_base = blockIdx.x * AU_BM;
+  // With clusters (size C along x) the C CTAs of a cluster share one row tile and deal its key tiles round-robin:
+  // rank r takes tiles r, r + C, ...; their partial (m, l, O) are merged through distributed shared memory at the end.
+  const int C = cluster > 1 ? cluster : 1;
+  const int rank = (int)(blockIdx.x % C);
+  const int row_base = (int)(blockIdx.x / C) * AU_BM;
   const int F = sd.F[b];
   const int n_c = (F + AU_BN - 1) / AU_BN, n_s = (Qn + AU_BN - 1) / AU_BN;
-  const int n_tiles = (row_base < rows_total) ? n_c + n_s : 0;     // a CTA past the last row does nothing
+  const int n_all = (row_base < rows_total) ? n_c + n_s : 0;       // a CTA past the last row does nothing
+  const int n_tiles = n_all > rank ? (n_all - rank + C - 1) / C : 0;   // this CTA's tiles; t below counts them
   const int ldq = n_heads * DH;
 
   if (warp < 4) {
@@ -161,8 +171,9 @@ k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ 
         }
         mbar_expect_tx(bar(s), 2 * AU_TILE);
         const uint32_t kd = smem_u32(KVs + (size_t)s * 2 * AU_TILE), vd = kd + AU_TILE;
-        const bool cache = t < n_c;
-        const int row = cache ? b * max_len + t * AU_BN : r0 + (t - n_c) * AU_BN;
+        const int gt = rank + t * C;                    // tile index in the sequence's key range
+        const bool cache = gt < n_c;
+        const int row = cache ? b * max_len + gt * AU_BN : r0 + (gt - n_c) * AU_BN;
         const CUtensorMap* mk = cache ? &map_ck : &map_sk;
         const CUtensorMap* mv = cache ? &map_cv : &map_sv;
         tma_load_2d(kd, mk, kvh * DH, row, bar(s));
@@ -235,7 +246,8 @@ k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ 
         break;
       }
       tc_fence_after();
-      const int valid_keys = (t < n_c) ? min(AU_BN, F - t * AU_BN) : min(AU_BN, Qn - (t - n_c) * AU_BN);
+      const int gt = rank + t * C;
+      const int valid_keys = (gt < n_c) ? min(AU_BN, F - gt * AU_BN) : min(AU_BN, Qn - (gt - n_c) * AU_BN);
       float sv[AU_BN];
 #pragma unroll
       for (int c = 0; c < AU_BN; c += 16) tc_ld16_nowait(lane_base + 128u + (uint32_t)(s * AU_BN + c), sv + c);
@@ -299,25 +311,92 @@ k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ 
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(8));               // P ready
     }
-    if (ok && n_tiles > 0 && mbar_wait(bar(9), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
-      tc_fence_after();
-      const int row = row_base + r;
-      const float inv = 1.f / l;
-      const bool valid = row < rows_total;
-      const int qi = valid ? row / G : 0, hg = valid ? row % G : 0;
-      uint4* dst = reinterpret_cast<uint4*>(out + (size_t)(r0 + qi) * ldq + (kvh * G + hg) * DH);
+    const bool have = ok && n_tiles > 0 && mbar_wait(bar(9), (uint32_t)(n_tiles - 1) & 1u, abort_flag);
+    if (have) tc_fence_after();
+    if (C == 1) {
+      if (have) {
+        const int row = row_base + r;
+        const float inv = 1.f / l;
+        const bool valid = row < rows_total;
+        const int qi = valid ? row / G : 0, hg = valid ? row % G : 0;
+        uint4* dst = reinterpret_cast<uint4*>(out + (size_t)(r0 + qi) * ldq + (kvh * G + hg) * DH);
+#pragma unroll 1
+        for (int c = 0; c < DH; c += 16) {
+          float v[16];
+          tc_ld16(lane_base + (uint32_t)c, v);
+          if (valid) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] *= inv;
+            dst[c >> 3] = pack8(v);
+            dst[(c >> 3) + 1] = pack8(v + 8);
+          }
+        }
+      }
+    } else {
+      // publish this CTA's partial result in its own shared memory (the K/V stages are idle by now):
+      // O as [16-column chunk][quarter][row][4 floats] (64 KB), then m and l per row
+      float4* po = reinterpret_cast<float4*>(KVs);
+      float* pm = reinterpret_cast<float*>(KVs + AU_BM * DH * 4);
 #pragma unroll 1
       for (int c = 0; c < DH; c += 16) {
         float v[16];
-        tc_ld16(lane_base + (uint32_t)c, v);
+        if (have) tc_ld16(lane_base + (uint32_t)c, v);
+        else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) po[((c >> 4) * 4 + i) * AU_BM + r] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+      }
+      pm[r] = have ? m_used : -INFINITY;
+      pm[AU_BM + r] = have ? l : 0.f;
+    }
+  }
+  if (C > 1) {
+    // Merge across the cluster: rank r finishes its share of the 16-column chunks for all 128 rows, combining the
+    // ranks' partials in rank order with the weights exp2(m_p - max_p m_p).  All threads of all CTAs reach both barriers.
+    cluster_sync();
+    if (warp < 4 && n_all > 0) {
+      const int r = threadIdx.x;
+      const int row = row_base + r;
+      const bool valid = row < rows_total;
+      const uint32_t base_o = smem_u32(KVs), base_m = base_o + AU_BM * DH * 4;
+      float wgt[8];
+      float mmax = -INFINITY;
+      for (int p = 0; p < C; ++p) {
+        wgt[p] = ld_cluster_f1(cluster_map(base_m + 4u * r, (unsigned)p));
+        mmax = fmaxf(mmax, wgt[p]);
+      }
+      float L = 0.f;
+      for (int p = 0; p < C; ++p) {
+        wgt[p] = (wgt[p] == -INFINITY) ? 0.f : ex2_approx(wgt[p] - mmax);
+        L += wgt[p] * ld_cluster_f1(cluster_map(base_m + 4u * (AU_BM + r), (unsigned)p));
+      }
+      const float inv = 1.f / L;
+      const int qi = valid ? row / G : 0, hg = valid ? row % G : 0;
+      uint4* dst = reinterpret_cast<uint4*>(out + (size_t)(r0 + qi) * ldq + (kvh * G + hg) * DH);
+      const int ch_lo = (DH / 16) * rank / C, ch_hi = (DH / 16) * (rank + 1) / C;
+      for (int ch = ch_lo; ch < ch_hi; ++ch) {
+        float v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        for (int p = 0; p < C; ++p) {
+          const uint32_t peer = cluster_map(base_o + (uint32_t)((ch * 4 * AU_BM + r) * 16), (unsigned)p);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float4 t4 = ld_cluster_f4(peer + (uint32_t)(i * AU_BM * 16));
+            v[4 * i] += wgt[p] * t4.x; v[4 * i + 1] += wgt[p] * t4.y; v[4 * i + 2] += wgt[p] * t4.z; v[4 * i + 3] += wgt[p] * t4.w;
+          }
+        }
         if (valid) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) v[i] *= inv;
-          dst[c >> 3] = pack8(v);
-          dst[(c >> 3) + 1] = pack8(v + 8);
+          dst[2 * ch] = pack8(v);
+          dst[2 * ch + 1] = pack8(v + 8);
         }
       }
     }
+    cluster_sync();
   }
   tc_fence_before();
   __syncthreads();

@@ -1,6 +1,7 @@
 // Host step driver and C ABI of the LSP decode library (see include/lsp.h for the contract).
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -35,7 +36,7 @@ struct lsp_ctx {
   int max_batch = 0, max_len = 0, max_rows = 0;
   size_t esz = 0;
   cudaStream_t stream = nullptr;
-  int gemm_impl = 1, attn_impl = 2, timing = 0, async_ops = 0, op_repeat = 1, op_rotate = 1, pdl = 1, attn_umma_min_rows = 384;
+  int gemm_impl = 1, attn_impl = 2, timing = 0, async_ops = 0, op_repeat = 1, op_rotate = 1, pdl = 1, attn_umma_min_rows = 0, attn_cluster = 1;
   // workspace carve (device)
   char *X = nullptr, *Nrm = nullptr, *Qb = nullptr, *Att = nullptr, *Hf = nullptr, *stage = nullptr;
   Top2* part = nullptr;
@@ -379,15 +380,26 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
       bool done = false;
 #ifndef LSP_NO_UMMA
       if constexpr (std::is_same<T, bf16>::value) {
-        // the tcgen05 kernel works on 128-row tiles: it pays from a few tiles per (sequence, KV head) upwards; below that
-        // the 64-row mma.sync kernel has more CTAs in flight
+        // the tcgen05 kernel (128-row tiles; with few CTAs the keys of a row tile are split over a cluster); a row-count
+        // threshold can send small passes to the 64-row mma.sync kernel instead
         if (c->attn_impl == 2 && dh == 128 && !c->attn_maps.empty() && maxQ * (m.n_heads / m.n_kv_heads) >= c->attn_umma_min_rows) {
           const int G = m.n_heads / m.n_kv_heads;
-          dim3 g3((maxQ * G + AU_BM - 1) / AU_BM, m.n_kv_heads, B);
+          const int row_tiles = (maxQ * G + AU_BM - 1) / AU_BM;
+          // few CTAs: split every row tile's keys over a cluster of 2, 4 or 8 CTAs (merged through DSMEM)
+          int cl = 1;
+          if (c->attn_cluster) {
+            int max_keys = 0;
+            for (int b = 0; b < B; ++b)
+              if (c->N[b] > 0) max_keys = std::max(max_keys, c->F[b] + c->pend[b] + (scattered ? c->G[b] : c->N[b]));
+            const int key_tiles = (max_keys + AU_BN - 1) / AU_BN;
+            const int ctas = row_tiles * m.n_kv_heads * B;
+            while (cl < 8 && 2 * cl * ctas <= c->umma.n_sm && 2 * cl <= key_tiles) cl *= 2;
+          }
+          dim3 g3(row_tiles * cl, m.n_kv_heads, B);
           const float sl2 = scale * 1.4426950408889634f;
           const CUtensorMap* mp = &c->attn_maps[4 * l];
-          launch_k(c->pdl, k_attn_umma, g3, dim3(AU_THREADS), (size_t)AU_SMEM, c->stream, mp[0], mp[1], mp[2], mp[3],
-                   (const bf16*)Qb, Att, sd, m.n_heads, m.n_kv_heads, c->max_len, sl2, c->d_status);
+          launch_k(c->pdl, k_attn_umma, g3, dim3(AU_THREADS), (size_t)AU_SMEM, c->stream, cl, mp[0], mp[1], mp[2], mp[3],
+                   (const bf16*)Qb, Att, sd, m.n_heads, m.n_kv_heads, c->max_len, sl2, cl, c->d_status);
           done = true;
         }
       }
@@ -667,6 +679,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   if (key == 0) c->gemm_impl = value;
   else if (key == 1) c->attn_impl = value;
   else if (key == 28) c->attn_umma_min_rows = value;
+  else if (key == 30) c->attn_cluster = value ? 1 : 0;
   else if (key == 2) c->timing = value;
   else if (key == 3) c->async_ops = value;
   else if (key == 4) c->op_repeat = value < 1 ? 1 : value;

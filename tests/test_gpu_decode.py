@@ -33,6 +33,8 @@ def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, 
         dec.set_option(0, impl)
     if attn_impl is not None:
         dec.set_option(1, attn_impl)
+        if attn_impl == 2:
+            dec.set_option(28, 0)          # the tcgen05 kernel at every row count, not only from its default threshold
     tokens = torch.zeros(1, P + G, dtype=torch.int32, device=DEV)
     tokens[0, :P] = prompt[0].to(DEV)
     dec.begin(tokens, [P], [G])
