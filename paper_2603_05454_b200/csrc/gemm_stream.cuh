@@ -627,7 +627,12 @@ int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn) {
   const long n_tiles = (NP + per_tile - 1) / per_tile;
   int mt;
   if (M <= UM_BM) mt = 1;
-  else if (M <= 2 * UM_BM) mt = st.stream_two_tiles == 1 ? 2 : (st.stream_two_tiles == 2 ? 1 : 0);
+  else if (M <= 2 * UM_BM) {
+    // layer GEMMs: two row tiles per CTA (each weight tile is used for all rows while it is in shared memory); the LM
+    // head has hundreds of column tiles, so two row groups of whole 128 x 256 tiles keep double-buffered accumulators
+    // and run 1.5 x faster there (the second row group finds its weight tile in L2)
+    mt = (Epi::kReduce && st.stream_two_tiles) ? 1 : (st.stream_two_tiles == 1 ? 2 : (st.stream_two_tiles == 2 ? 1 : 0));
+  }
   else if (st.stream_big_mt != 3) mt = st.stream_big_mt;   // 0 = leave large problems to the tiled kernel
   else {
     // 256 x 256 tiles (two row tiles per CTA) move a third less operand data through L2 per flop than 128 x 256 ones and
