@@ -39,15 +39,33 @@ CLASSES = ("misc", "gemm", "attn", "head", "scan", "commit")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures summarised under
-# profiles/, keyed by kernel class, with the hash of the kernel sources they were taken on.  A class whose sources
-# changed since reports null.
-NCU_TRAFFIC = {}
+# profiles/, keyed by kernel class: the captured launch's traffic and algorithmic bytes, and the hash of the kernel
+# sources the capture was taken on.  The class's launches differ in shape, and traffic grows in proportion to the
+# weight bytes streamed, so the reported figure is the class's mean algorithmic bytes per launch scaled by the
+# captured ratio.  A class whose sources changed since the capture reports null.
+CLASS_SOURCES = {
+    "gemm": ("gemm_stream.cuh", "gemm_umma.cuh", "epilogues.cuh", "common.cuh"),
+    "head": ("gemm_stream.cuh", "gemm_umma.cuh", "epilogues.cuh", "common.cuh"),
+    "attn": ("attention_umma.cuh", "common.cuh"),
+    "commit": ("misc_kernels.cuh", "common.cuh"),
+}
+NCU_TRAFFIC = {
+    # k_gemm_stream<128,1,1,EpiStore>, M 64, N 12288, K 4096: profiles/k_gemm_stream_M64_N12288_K4096.md
+    "gemm": {"captured_bytes": 105.0e6, "algorithmic_bytes": 102.8e6, "src": "a8028268591d"},
+    # k_gemm_stream<256,1,1,EpiHead>, 64 rows: profiles/k_gemm_stream_head_M64_V126464.md
+    "head": {"captured_bytes": 1062.2e6, "algorithmic_bytes": 1037.0e6, "src": "a8028268591d"},
+    # k_attn_umma, 16 x (128 query rows over 2048 keys): profiles/k_attn_umma_B16_F1920.md
+    "attn": {"captured_bytes": 571.6e6, "algorithmic_bytes": 570.4e6, "src": "98c8e2d8410f"},
+    # k_commit_append of a 16 x 1920-row prompt block: profiles/k_commit_append_prompt_B16_P1920.md
+    "commit": {"captured_bytes": 1969.0e6, "algorithmic_bytes": 2013.3e6, "src": "c62d33c71cc9"},
+}
 
 
-def source_hash():
+def source_hash(name=None):
     h = hashlib.sha1()
     d = os.path.join(ROOT, "paper_2603_05454_b200", "csrc")
-    for f in sorted(os.listdir(d)):
+    files = CLASS_SOURCES.get(name) or sorted(os.listdir(d))
+    for f in files:
         h.update(open(os.path.join(d, f), "rb").read())
     return h.hexdigest()[:12]
 
@@ -214,7 +232,6 @@ def class_report(cnt, tms, peaks):
     """Per-class achieved bandwidth / throughput from the library's work counters and per-launch event times."""
     hbm = peaks["hbm_gbs"]
     tc = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
-    src = source_hash()
     out = {}
     work = {"gemm": (cnt["gemm_bytes"], cnt["gemm_flops"]), "attn": (cnt["attn_bytes"], cnt["attn_flops"]),
             "head": (cnt["head_bytes"], cnt["head_flops"]), "commit": (cnt["append_bytes"], 0.0)}
@@ -231,7 +248,9 @@ def class_report(cnt, tms, peaks):
                 e["tensor_frac_sustained"] = round(e["tflops"] / tc, 4)
             e["bytes_per_launch"] = round(b / n) if n else None
         t = NCU_TRAFFIC.get(name)
-        e["traffic"] = t["bytes_per_launch"] if t and t.get("src") == src else None
+        e["traffic"] = None
+        if t and n and name in work and t.get("src") == source_hash(name):
+            e["traffic"] = round(work[name][0] / n * t["captured_bytes"] / t["algorithmic_bytes"])
         out[name] = e
     return out
 
