@@ -16,6 +16,8 @@ Prints ONE JSON line:
   classes        the same figures for every kernel class (attention, LM head, append, ...)
   cpu_baseline   the CPU oracle timed on a bounded sample of the same workload (rank 0, N = 1 only)
   also           a shorter run of the Dream-7B-shaped decode (cfg4), whose passes are tensor-bound
+  adaptive_tau   the same workload decoded in the adaptive-threshold mode (Eq. 2, block in [0.25 N, 0.50 N]): passes,
+                 suffix length per pass (geometric decay), rows touched in total against the G/beta..G/alpha bounds
 
 `--impl reference` times the CPU oracle alone (there is no other reference implementation of this path).
 With N > 1 (torchrun) every rank runs an independent replica of the workload with its own prompts: the path has
@@ -255,7 +257,45 @@ def class_report(cnt, tms, peaks):
     return out
 
 
-def run_decode_bench(wl, dev, rank, world, peaks, steps, warmup, sampler=None, with_e2e=True):
+def run_adaptive_leg(dec, wl, bm, tokens, Pl, Gl, steps, barrier):
+    """The same resident decoder in the adaptive-threshold mode (Eq. 2; block size kept within [alpha N, beta N],
+    alpha = 0.25, beta = 0.50, snap window 16): the active suffix then shrinks geometrically, so a decode takes
+    O(log G) denoiser passes and touches O(G) rows in total instead of O(G^2)."""
+    import numpy as np
+    import torch
+    from paper_2603_05454_b200 import SchedCfg
+    B, G = wl.batch, wl.gen_len
+    alpha, beta = 0.25, 0.50
+    dec.set_sched(SchedCfg(mode=1, tau=wl.tau, alpha=alpha, beta=beta, delim_bitmap=bm))
+    for _ in range(2):
+        dec.begin(tokens, Pl, Gl)
+        dec.generate()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    passes = 0
+    for _ in range(steps):
+        dec.begin(tokens, Pl, Gl)
+        passes += dec.generate()[0]
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    dec.begin(tokens, Pl, Gl)
+    n, recs = dec.generate(max_recs=B * (G + 1))
+    n_before = [int(np.mean([r["n_before"] for r in recs[i:i + B]])) for i in range(0, len(recs), B)]
+    masked_rows = sum(r["n_before"] for r in recs)
+    ratios = [n_before[i + 1] / n_before[i] for i in range(len(n_before) - 1) if n_before[i] >= 32]
+    out = {"alpha": alpha, "beta": beta, "snap_window": 16, "value": B * G * steps / (ms * 1e-3), "unit": "tokens/s",
+           "ms_per_decode": ms / steps, "denoiser_passes_per_decode": passes / steps,
+           "masked_suffix_per_pass_mean_over_batch": n_before,
+           "suffix_ratio_per_pass_while_at_least_32": [round(x, 3) for x in ratios],
+           "masked_rows_total_per_sequence": masked_rows / B,
+           "bounds_G_over_beta_G_over_alpha": [G / beta, G / alpha], "quadratic_G2_over_2": G * G / 2}
+    dec.set_sched(SchedCfg(tau=wl.tau, delim_bitmap=bm))
+    return out
+
+
+def run_decode_bench(wl, dev, rank, world, peaks, steps, warmup, sampler=None, with_e2e=True, adaptive=False):
     import numpy as np
     import torch
     import lsp_synth as S
@@ -339,6 +379,8 @@ def run_decode_bench(wl, dev, rank, world, peaks, steps, warmup, sampler=None, w
     res["step_ms_by_rows"] = {str(k): round(float(np.median(rows_ms[k])), 4) for k in pick}
     live = [r["L_commit"] for r in recs if r["n_before"] > 0]
     res["l_commit_mean"] = float(np.mean(live)) if live else None
+    if adaptive:
+        res["adaptive"] = run_adaptive_leg(dec, wl, bm, tokens, Pl, Gl, steps, barrier)
     dec.close()
     del dec, w
     torch.cuda.empty_cache()
@@ -517,7 +559,7 @@ def main():
                 "topologies": cmp_, "gpu_launches": lsp["gpu_launches"], "clocks": clocks}
         print(json.dumps(line))
         return 0
-    r = run_decode_bench(wl, dev, rank, world, peaks, args.steps, args.warmup, sampler)
+    r = run_decode_bench(wl, dev, rank, world, peaks, args.steps, args.warmup, sampler, adaptive=(world == 1))
     (ms_max, e2e_max), tokens_total = reduce_replicas([r["ms"], r.get("e2e_ms", 0.0)], r["tokens"], world, dev)
     value = tokens_total / (ms_max * 1e-3)
     gemm = r["classes"]["gemm"]
@@ -544,6 +586,8 @@ def main():
             "e2e": {"value": tokens_total / (e2e_max * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": r["h2d"],
                     "d2h_bytes_per_step": r["d2h"]},
             "gpu_launches": r["launches"], "clocks": r["clocks"]}
+    if r.get("adaptive"):
+        line["adaptive_tau"] = r["adaptive"]
 
     if rank == 0 and world == 1 and args.also != "none" and args.also != args.workload:
         wl2 = S.config(args.also)

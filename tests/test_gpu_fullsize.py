@@ -81,3 +81,46 @@ def test_full_width_layer_teacher_forced_steps(name):
     # fixed-k policy then walks the row count down through the one-row-tile regime
     _teacher_forced(sh, 21, 50, 250, SchedCfg(tau=0.9), (1, 64), max_steps=2)
     _teacher_forced(sh, 22, 8, 150, SchedCfg(mode=2, fixed_k=60), (1, 64), max_steps=3)
+
+
+def test_full_width_layer_teacher_forced_steps_adaptive_threshold():
+    """Eq. 2 at full layer width: the adaptive block keeps L' inside [alpha N, beta N], step by step against the oracle."""
+    from paper_2603_05454_b200 import SchedCfg
+    sh = S.ModelShape(1, 4096, 32, 32, 128, 12288, 8192, dtype="bf16", head_scale=4.0)
+    _teacher_forced(sh, 23, 40, 260, SchedCfg(mode=1, alpha=0.25, beta=0.5), (1, 64), max_steps=4)
+
+
+def test_adaptive_threshold_decode_shrinks_the_suffix_geometrically_at_full_vocabulary():
+    """Properties of Eq. 2 that hold at any size, on a free-running decode (two full-width LLaDA-shaped layers, the full
+    126464-entry vocabulary, batch 2, 64 + 512): every step's run lies in [ceil(alpha N), floor(beta N)], the committed
+    block is the run or a delimiter at most W before it, the suffix therefore shrinks by a constant factor while
+    alpha N > W, and the rows touched in total stay far below the quadratic count of one-token steps."""
+    import math
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+    alpha, beta, W = 0.25, 0.5, 16
+    sh = S.ModelShape(2, 4096, 32, 32, 128, 12288, 126464, dtype="bf16", head_scale=12.0)
+    w = S.make_weights(sh, 5, device=DEV)
+    bm = S.delimiter_bitmap(sh.vocab, 1, 32).to(DEV)
+    B, P, G = 2, 64, 512
+    dec = LSPDecoder(sh, w, SchedCfg(mode=1, alpha=alpha, beta=beta, snap_window=W, delim_bitmap=bm), B, P + G, device=DEV)
+    tokens = torch.full((B, P + G), sh.mask_id, dtype=torch.int32, device=DEV)
+    tokens[:, :P] = S.make_prompt(B, P, sh, 9).to(DEV)
+    dec.begin(tokens, [P] * B, [G] * B)
+    n, recs = dec.generate(max_recs=B * (G + 1))
+    dec.close()
+    assert int((tokens == sh.mask_id).sum()) == 0
+    for b in range(B):
+        mine = [r for r in recs[b::B] if r["n_before"] > 0]
+        N = G
+        for r in mine:
+            assert r["n_before"] == N
+            lo = max(1, math.ceil(alpha * N))
+            hi = min(N, max(lo, math.floor(beta * N)))
+            assert lo <= r["L_run"] <= hi, r
+            assert max(1, r["L_run"] - W) <= r["L_commit"] <= r["L_run"], r
+            if alpha * N > 2 * W:                          # the block is at least half the lower end of the range
+                assert N - r["L_commit"] <= (1 - alpha / 2) * N
+            N -= r["L_commit"]
+        assert N == 0
+        assert sum(r["n_before"] for r in mine) < G * G / 8     # one-token steps would touch G (G + 1) / 2 masked rows
+    assert n == max(len([r for r in recs[b::B] if r["n_before"] > 0]) for b in range(B))
