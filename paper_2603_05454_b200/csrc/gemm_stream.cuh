@@ -40,6 +40,8 @@ struct StreamArgs {
   int whole_tiles;  // 1: shares are whole tiles (no tile is split between CTAs)
   int cluster;      // > 1: the launch uses thread block clusters of this size, one cluster per tile, CTA rank r owning the
                     // r-th K slice; the partial tiles are then reduced through distributed shared memory (see the kernel)
+  int cl_rounds;    // ... in this many rounds: 1 = the whole partial tile at once, MT = one row tile (128 rows) at a time,
+                    // for partial tiles larger than the pipeline's shared memory
   int kc;           // K chunks (one per stage) per tile
   int a_rows;       // activation box rows (M rounded up to a multiple of 8)
   int atoms;        // 64-element K atoms per stage (1 or 2)
@@ -71,7 +73,7 @@ __device__ __forceinline__ uint32_t cluster_map(uint32_t saddr, unsigned rank) {
 }
 __device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
   float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
   return v;
 }
 
@@ -355,8 +357,11 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         float4* slot_base = args.cluster > 1
                                 ? reinterpret_cast<float4*>(smem)
                                 : reinterpret_cast<float4*>(args.scratch + (size_t)(g * 2 + (seg == 0 ? 0 : 1)) * ROWS * BN);
+        // with several cluster rounds only the first row tile is published here; the others stay in tensor memory
+        const bool by_tile = args.cluster > 1 && args.cl_rounds > 1;
+        const int PR = by_tile ? UM_BM : ROWS;          // rows of the published partial
 #pragma unroll 1
-        for (int mt = 0; mt < MT; ++mt) {
+        for (int mt = 0; mt < (by_tile ? 1 : MT); ++mt) {
           const int m = mt * UM_BM + r_in;              // row within the row group
 #pragma unroll 1
           for (int c = 0; c < BN; c += 16) {
@@ -371,7 +376,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             if (row0 + m < args.M) {
 #pragma unroll
               for (int i = 0; i < 4; ++i)
-                slot_base[(size_t)((c >> 4) * 4 + i) * ROWS + m] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                slot_base[(size_t)((c >> 4) * 4 + i) * PR + m] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
             }
           }
         }
@@ -475,46 +480,81 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     // result does not depend on timing) straight from their shared memory, and runs the fused epilogue on them.
     // Every thread of every CTA reaches both barriers (no early exits above), so they cannot hang.
     const int C = args.cluster;
-    cluster_sync();
-    if constexpr (!Epi::kReduce) {
-      if (warp >= 2 && warp <= 5 && n_units > 0) {
-        constexpr int CH = Epi::kDual ? HALF : BN;
-        constexpr int NCH = CH / 16;
-        const unsigned rank = cluster_ctarank();
-        const int ch_lo = NCH * (int)rank / C, ch_hi = NCH * ((int)rank + 1) / C;
-        const int rows_here = min(ROWS, args.M - cl_row0);
-        const int n_items = rows_here * (ch_hi - ch_lo);
-        const uint32_t base = smem_u32(smem);
-        for (int idx = threadIdx.x - 64; idx < n_items; idx += 128) {
-          const int mm = idx % rows_here, ch = ch_lo + idx / rows_here, c = ch * 16;
-          float a0[16], a1[16];
+    const int rounds = args.cl_rounds > 1 ? MT : 1;
+    const int PR = rounds > 1 ? UM_BM : ROWS;            // rows of the partial published per round
+#pragma unroll 1
+    for (int rd = 0; rd < rounds; ++rd) {
+      if (rd > 0 && warp >= 2 && warp <= 5 && n_units > 0) {
+        // publish the next row tile (a cluster CTA has a single segment: accumulator set 0, ACC = 1 with two row tiles)
+        const int q = warp & 3, r_in = q * 32 + lane;
+        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+        float4* slot_base = reinterpret_cast<float4*>(smem);
+        tc_fence_after();
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 16) {
+          float v[16];
+          tc_ld16(t_row + rd * ACC * BN + c, v);
+          if (cl_row0 + rd * UM_BM + r_in < args.M) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
-          const uint32_t off0 = (uint32_t)(((c >> 4) * 4 * ROWS + mm) * 16);
-          const uint32_t off1 = (uint32_t)((((HALF + c) >> 4) * 4 * ROWS + mm) * 16);
-          for (int pr = 0; pr < C; ++pr) {
-            const uint32_t peer = cluster_map(base, (unsigned)pr);
-            float4 t0[4], t1[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) t0[i] = ld_cluster_f4(peer + off0 + (uint32_t)(i * ROWS * 16));
-            if (Epi::kDual) {
-#pragma unroll
-              for (int i = 0; i < 4; ++i) t1[i] = ld_cluster_f4(peer + off1 + (uint32_t)(i * ROWS * 16));
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              a0[4 * i] += t0[i].x; a0[4 * i + 1] += t0[i].y; a0[4 * i + 2] += t0[i].z; a0[4 * i + 3] += t0[i].w;
-              if (Epi::kDual) {
-                a1[4 * i] += t1[i].x; a1[4 * i + 1] += t1[i].y; a1[4 * i + 2] += t1[i].z; a1[4 * i + 3] += t1[i].w;
-              }
-            }
+            for (int i = 0; i < 4; ++i)
+              slot_base[(size_t)((c >> 4) * 4 + i) * PR + r_in] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
           }
-          const int j0 = cl_tile * CH;
-          if (j0 + c < args.n_pairs) epi16(epi, cl_row0 + mm, j0 + c, a0, a1);
         }
       }
+      cluster_sync();
+      if constexpr (!Epi::kReduce) {
+        if (warp >= 2 && warp <= 5 && n_units > 0) {
+          constexpr int CH = Epi::kDual ? HALF : BN;
+          constexpr int NCH = CH / 16;
+          const unsigned rank = cluster_ctarank();
+          const int ch_lo = NCH * (int)rank / C, ch_hi = NCH * ((int)rank + 1) / C;
+          const int r_first = cl_row0 + rd * PR;                       // first activation row of this round
+          const int rows_here = max(0, min(PR, args.M - r_first));
+          const int n_items = rows_here * (ch_hi - ch_lo);
+          const uint32_t base = smem_u32(smem);
+          for (int idx = threadIdx.x - 64; idx < n_items; idx += 128) {
+            const int mm = idx % rows_here, ch = ch_lo + idx / rows_here, c = ch * 16;
+            float a0[16], a1[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
+            const uint32_t off0 = (uint32_t)(((c >> 4) * 4 * PR + mm) * 16);
+            const uint32_t off1 = (uint32_t)((((HALF + c) >> 4) * 4 * PR + mm) * 16);
+            // up to four ranks' pieces are requested before any is added (the loads are independent; the sum stays in
+            // rank order)
+            for (int pb = 0; pb < C; pb += 4) {
+              float4 t0[4][4], t1[4][4];
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                if (pb + x < C) {
+                  const uint32_t peer = cluster_map(base, (unsigned)(pb + x));
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) t0[x][i] = ld_cluster_f4(peer + off0 + (uint32_t)(i * PR * 16));
+                  if (Epi::kDual) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) t1[x][i] = ld_cluster_f4(peer + off1 + (uint32_t)(i * PR * 16));
+                  }
+                }
+              }
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                if (pb + x < C) {
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    a0[4 * i] += t0[x][i].x; a0[4 * i + 1] += t0[x][i].y; a0[4 * i + 2] += t0[x][i].z; a0[4 * i + 3] += t0[x][i].w;
+                    if (Epi::kDual) {
+                      a1[4 * i] += t1[x][i].x; a1[4 * i + 1] += t1[x][i].y; a1[4 * i + 2] += t1[x][i].z; a1[4 * i + 3] += t1[x][i].w;
+                    }
+                  }
+                }
+              }
+            }
+            const int j0 = cl_tile * CH;
+            if (j0 + c < args.n_pairs) epi16(epi, r_first + mm, j0 + c, a0, a1);
+          }
+        }
+      }
+      cluster_sync();      // nobody overwrites its partial, or leaves, while a peer may still read its shared memory
     }
-    cluster_sync();      // nobody leaves while a peer may still read its shared memory
   }
   tc_fence_before();
   __syncthreads();
@@ -533,14 +573,23 @@ inline size_t stream_scratch_bytes(int n_ctas, int bn, int mt) { return (size_t)
 // With at most as many tiles as SMs, a grid that is a multiple of the tile count splits each tile into equal K slices
 // instead (no split at all when there are more than half as many tiles as SMs).  Measured on the LLaDA layer shapes
 // the second choice is as fast or faster at every row count from 2 to 128, so it is the default.
-inline int stream_grid(const UmmaState& st, int n_tiles, int M) {
-  if (st.target_ctas > 0) return st.target_ctas;
-  int splits = n_tiles <= st.n_sm ? st.n_sm / n_tiles : 0;
-  if (st.stream_cluster && splits > 1) {          // a split of 2, 4 or 8 can run as a thread block cluster
-    int p2 = 1;
-    while (2 * p2 <= splits && 2 * p2 <= 8) p2 *= 2;
+// K slices per tile when the tiles are fewer than the SMs.  With clusters on: a power of two up to 8 (a cluster of 3
+// measured 40 % slower than the same split without clusters), and no more clusters than can be resident at once
+// (sixteen clusters of 8 do not fit the 148 SMs' GPC layout: the launch would run in two waves).
+inline int stream_splits(const UmmaState& st, long n_tiles) {
+  int splits = n_tiles <= st.n_sm ? (int)(st.n_sm / n_tiles) : 0;
+  if (st.stream_cluster && splits > 1) {
+    int p2 = 1, lg = 0;
+    while (2 * p2 <= splits && 2 * p2 <= 8) { p2 *= 2; ++lg; }
+    while (p2 > 1 && n_tiles > st.max_clusters[lg]) { p2 /= 2; --lg; }
     splits = p2;
   }
+  return splits;
+}
+
+inline int stream_grid(const UmmaState& st, int n_tiles, int M) {
+  if (st.target_ctas > 0) return st.target_ctas;
+  const int splits = stream_splits(st, n_tiles);
   const int aligned = splits > 0 ? n_tiles * splits : st.n_sm;
   if (st.stream_grid_mode == 1) return st.n_sm;
   if (st.stream_grid_mode == 2) return aligned;
@@ -573,6 +622,29 @@ inline StreamShape stream_shape(const UmmaState& st, int a_rows, int bn, int mt,
 // Activation box rows: all rows (rounded up to 8) when they fit one group of 128 mt rows, else a full group.
 inline int stream_a_rows(int M, int mt) { return M <= UM_BM * mt ? (M + 7) / 8 * 8 : UM_BM * mt; }
 
+// Asks the runtime how many clusters of 2, 4 and 8 CTAs of the streaming kernel (one CTA per SM) can be resident at once.
+inline void stream_query_clusters(UmmaState& st) {
+  auto kern = k_gemm_stream<128, 1, 1, EpiStore<bf16>>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, st.max_smem) != cudaSuccess) return;
+  st.max_clusters[0] = st.n_sm;
+  for (int lg = 1; lg <= 3; ++lg) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(8 * st.n_sm);
+    cfg.blockDim = dim3(ST_THREADS);
+    cfg.dynamicSmemBytes = (size_t)st.max_smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1u << lg;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0) st.max_clusters[lg] = n;
+  }
+  cudaGetLastError();
+}
+
 template <int BN, int MT, int NI, typename Epi>
 int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
                   int n_rows_w, const Epi& epi, unsigned* status, int box_rows) {
@@ -601,15 +673,17 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
   int grid = whole ? st.n_sm : stream_grid(st, (int)T, M);
   if (grid > T * kc) grid = (int)(T * kc);
   // K slices of one tile on the CTAs of one cluster: the reduction then stays on chip
-  int cluster = 0;
+  int cluster = 0, cl_rounds = 1;
   if (!whole && !Epi::kReduce && st.stream_cluster && grid % T == 0) {
     const int splits = (int)(grid / T);
     // sizes 2, 4 and 8 only: a cluster of 3 measured 40 % slower than the same split without clusters
-    if ((splits == 2 || splits == 4 || splits == 8) && kc >= splits &&
-        (size_t)sh.stages * sh.stage_bytes >= (size_t)UM_BM * MT * BN * sizeof(float))
+    const size_t area = (size_t)sh.stages * sh.stage_bytes, tile_bytes = (size_t)UM_BM * BN * sizeof(float);
+    if ((splits == 2 || splits == 4 || splits == 8) && kc >= splits && area >= tile_bytes) {
       cluster = splits;
+      if (area < MT * tile_bytes) cl_rounds = MT;      // the partial tile is published one row tile at a time
+    }
   }
-  StreamArgs args{M, NP, n_tiles, row_groups, whole, cluster, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch,
+  StreamArgs args{M, NP, n_tiles, row_groups, whole, cluster, cl_rounds, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch,
                   st.counters, status};
   cudaError_t e = launch_k(st.pdl, k_gemm_stream<BN, MT, NI, Epi>, dim3(grid), dim3(ST_THREADS), smem, stream, cluster, *ma, *mb0,
                            *mb1, args, epi);
@@ -635,13 +709,19 @@ int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn) {
   }
   else if (st.stream_big_mt != 3) mt = st.stream_big_mt;   // 0 = leave large problems to the tiled kernel
   else {
-    // 256 x 256 tiles (two row tiles per CTA) move a third less operand data through L2 per flop than 128 x 256 ones and
-    // measure about 12 % faster when both fill the SMs equally well; otherwise the fuller last wave wins
-    auto wave_eff = [&](int m) {
-      const long t = n_tiles * ((M + UM_BM * m - 1) / (UM_BM * m));
-      return (double)t / (double)((t + st.n_sm - 1) / st.n_sm * st.n_sm);
+    // 256 x 256 tiles (two row tiles per CTA) need a third less operand data per flop than 128 x 256 ones, which the
+    // SM's shared-memory fill rate cannot quite sustain: they measure about 1.25 x faster when both fill the SMs equally
+    // well.  Otherwise the better-filled grid wins; few tiles count with the K split their cluster would get, and rows
+    // that only pad the last row group count as waste.
+    auto fill = [&](int m) {
+      const long groups = (M + UM_BM * m - 1) / (UM_BM * m);
+      const long t = n_tiles * groups;
+      long ctas = t;
+      if (t < st.n_sm && st.stream_cluster && !Epi::kReduce) ctas = t * stream_splits(st, t);
+      const double waves = (double)((ctas + st.n_sm - 1) / st.n_sm * st.n_sm);
+      return (double)ctas / waves * (double)M / (double)(groups * UM_BM * m);
     };
-    mt = (2 * bn <= 512 && 1.12 * wave_eff(2) > wave_eff(1)) ? 2 : 1;
+    mt = (2 * bn <= 512 && 1.25 * fill(2) > fill(1)) ? 2 : 1;
   }
   if (mt == 0 || mt * bn > 512) return 0;
   const int row_groups = (M + UM_BM * mt - 1) / (UM_BM * mt);

@@ -638,6 +638,7 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
       lsp_destroy(c);
       return LSP_ERR_CUDA;
     }
+    stream_query_clusters(c->umma);
     if (model->head_dim == 128) {
       // tensor maps of the K / V planes for the tcgen05 attention kernel
       const int kvd = model->n_kv_heads * model->head_dim;
@@ -1065,7 +1066,7 @@ int lsp_linear_static(const void* A, const void* W, void* out, int M, int N, int
     static_msg(err, err_len, "lsp_linear_static: clearing the counters failed (%s)", cudaGetErrorString(e));
     return LSP_ERR_CUDA;
   }
-  StreamArgs args{M, N, n_tiles, 1, 0, 0, kc, a_rows, atoms, kStaticBN / 2, stages, partials, counters, status};
+  StreamArgs args{M, N, n_tiles, 1, 0, 0, 1, kc, a_rows, atoms, kStaticBN / 2, stages, partials, counters, status};
   EpiStore<bf16> epi{(bf16*)out, N};
   k_gemm_stream<kStaticBN, 1, 2, EpiStore<bf16>><<<grid, ST_THREADS, smem, stream>>>(ma, mb, mb, args, epi);
   e = cudaGetLastError();

@@ -90,3 +90,42 @@ def test_linear_bf16_weight_streaming_kernel(grid_mode, shape):
     ref = g / (1 + np.exp(-g)) * u
     np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05)
     dec.close()
+
+
+@pytest.mark.parametrize("case", [
+    # (M, N, K, options): 256 x 256 tiles whose K slices run as one cluster; the fp32 partial tile (256 KB) is larger
+    # than the pipeline's shared memory, so it is reduced one row tile at a time
+    (200, 4096, 4096, {20: 256}), (256, 12288, 4096, {20: 256}), (130, 4096, 12288, {20: 256}),
+    (640, 4096, 12288, {}), (1000, 3584, 3584, {}), (300, 2048, 1024, {}), (257, 512, 2048, {}),
+    (640, 4096, 4096, {29: 0}),
+])
+def test_linear_bf16_cluster_split_of_two_row_tiles(case):
+    M, N, K, opts = case
+    tdt = torch.bfloat16
+    dec = _dec("bf16")
+    for k, v in opts.items():
+        dec.set_option(k, v)
+    A = S.normal((M, K), 3, 1, 1.0, tdt, DEV)
+    W = S.normal((N, K), 3, 2, 0.05, tdt, DEV)
+    W2 = S.normal((N, K), 3, 3, 0.05, tdt, DEV)
+    X0 = S.normal((M, N), 3, 4, 1.0, tdt, DEV)
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    a, w, w2, x0 = f64(A), f64(W), f64(W2), f64(X0)
+    rtol = 1.0 / 128
+    out = torch.empty(M, N, dtype=tdt, device=DEV)
+    outs = []
+    for rep in range(2):
+        dec.op_linear(0, A, W, None, out)
+        ref = a @ w.T
+        np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05)
+        outs.append(out.clone())
+    assert torch.equal(outs[0], outs[1])       # rank-order summation: the same bits every time
+    xr = X0.clone()
+    dec.op_linear(1, A, W, None, xr)
+    ref = x0 + a @ w.T
+    np.testing.assert_allclose(f64(xr), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05)
+    dec.op_linear(2, A, W, W2, out)
+    g, u = a @ w.T, a @ w2.T
+    ref = g / (1 + np.exp(-g)) * u
+    np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05)
+    dec.close()
