@@ -315,11 +315,9 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         for (int mt = 0; mt < MT; ++mt) {
           const int m = row0 + mt * UM_BM + r_in;
           Top2 red = top2_empty();
-#pragma unroll 1
-          for (int c = 0; c < CH; c += 16) {
-            float a0[16], a1[16];
-            tc_ld16(t_row + mt * ACC * BN + c, a0);
-            if (Epi::kDual) tc_ld16(t_row + mt * ACC * BN + HALF + c, a1);
+          // one chunk of 16 columns (or pairs) at a time; the next chunk's tensor-memory loads are in flight while this
+          // one is converted and stored (with K-parity accumulators the extra loads are not pipelined)
+          auto consume = [&](int c, float (&a0)[16], float (&a1)[16]) {
             if constexpr (ACC == 2) {               // add the second K-parity accumulator
               float b0[16];
               tc_ld16(t_row + BN + c, b0);
@@ -340,6 +338,25 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             } else {
               if (m < args.M && j0 + c < args.n_pairs) epi16(epi, m, j0 + c, a0, a1);
             }
+          };
+          auto request = [&](int c, float (&a0)[16], float (&a1)[16]) {
+            tc_ld16_nowait(t_row + mt * ACC * BN + c, a0);
+            if (Epi::kDual) tc_ld16_nowait(t_row + mt * ACC * BN + HALF + c, a1);
+          };
+          float p0[16], p1[16], q0[16], q1[16];
+          request(0, p0, p1);
+#pragma unroll 1
+          for (int c = 0; c < CH; c += 32) {
+            tc_wait_ld();
+            tc_pin16(p0);
+            if (Epi::kDual) tc_pin16(p1);
+            request(c + 16, q0, q1);
+            consume(c, p0, p1);
+            tc_wait_ld();
+            tc_pin16(q0);
+            if (Epi::kDual) tc_pin16(q1);
+            if (c + 32 < CH) request(c + 32, p0, p1);
+            consume(c + 16, q0, q1);
           }
           if constexpr (Epi::kReduce) {
             if (m < args.M) epi.part[(size_t)m * epi.n_tiles + tile] = red;
