@@ -219,7 +219,7 @@ int lsp_op_linear(lsp_ctx* ctx, int op, const void* A, const void* W, const void
 
 /* Device time (ms) accumulated since lsp_reset_counters() by kernel class, host float[8]:
  * 0 embed+norms, 1 layer GEMMs, 2 attention, 3 fused LM head, 4 merge+scan, 5 commit/append, 6 whole steps
- * (always filled), 7 reserved.  Classes 0-5 are only filled while option key 2 (per-class CUDA-event timing)
+ * (always filled), 7 host time spent queueing those steps' launches (always filled).  Classes 0-5 are only filled while option key 2 (per-class CUDA-event timing)
  * is 1.  Synchronises the stream. */
 int lsp_last_timing(lsp_ctx* ctx, float* ms);
 

@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <chrono>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -327,6 +328,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   h[3 * s + B] = M;
   h[4 * s + B] = Mh;
   if (M == 0) return fail(c, LSP_ERR_STATE, "lsp_denoise_step: every sequence is already fully committed");
+  const auto host_t0 = std::chrono::steady_clock::now();
   CU(cudaEventRecord(c->ev0, c->stream));
   CU(cudaMemcpyAsync(c->d_desc, h, 7 * (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
   const StepDesc sd = desc_of(c);
@@ -464,6 +466,8 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   c->counters[CNT_STEPS] += 1;
   if (rc) return rc;
   CU(cudaEventRecord(c->ev1, c->stream));
+  // host time spent queueing the pass (everything between the two event records)
+  c->timing_ms[7] += std::chrono::duration<float, std::milli>(std::chrono::steady_clock::now() - host_t0).count();
   CU(cudaStreamSynchronize(c->stream));
   seg_collect(c);
   rc = check_status(c);

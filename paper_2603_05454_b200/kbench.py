@@ -126,12 +126,14 @@ def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False, opts=
         return n
 
     run()
+    dec.reset_counters()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     n_plain = run()
     e1.record()
     torch.cuda.synchronize()
     plain_ms = e0.elapsed_time(e1)
+    tp = dec.last_timing()          # plain run: device time of the passes and host time spent queueing them
     dec.set_option(2, 1)
     dec.reset_counters()
     n = 0
@@ -143,7 +145,8 @@ def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False, opts=
     names = ("misc", "gemm", "attn", "head", "scan", "commit")
     return dict(workload=name, passes=n, ms_per_pass_plain=round(plain_ms / n_plain, 4),
                 ms_per_pass={k: round(float(t[i]) / n, 4) for i, k in enumerate(names)},
-                ms_per_pass_total=round(float(t[6]) / n, 4), launches_per_pass=c["launches"] / n,
+                ms_per_pass_total=round(float(t[6]) / n, 4), ms_per_pass_plain_device=round(float(tp[6]) / n_plain, 4),
+                host_queue_ms_per_pass_plain=round(float(tp[7]) / n_plain, 4), launches_per_pass=c["launches"] / n,
                 gemm_gbs=round(c["gemm_bytes"] / (float(t[1]) * 1e6), 1),
                 gemm_tflops=round(c["gemm_flops"] / (float(t[1]) * 1e9), 1),
                 attn_gbs=round(c["attn_bytes"] / (float(t[2]) * 1e6), 1),
