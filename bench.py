@@ -275,7 +275,7 @@ def run_gemm_chain(dec, w, sh, M, dev, reps=3):
     dec.set_option(3, 1)                                   # queue only; no synchronisation per call
 
     def chain():
-        for lw in w["layers"]:
+        for lw in dec.layer_weights:
             dec.op_linear(0, a_d, lw["w_qkv"], None, o_qkv)
             dec.op_linear(1, a_q, lw["w_o"], None, x)
             dec.op_linear(2, a_d, lw["w_gate"], lw["w_up"], h_f)
@@ -291,7 +291,7 @@ def run_gemm_chain(dec, w, sh, M, dev, reps=3):
     ev1.record()
     torch.cuda.synchronize(dev)
     dec.set_option(3, 0)
-    dec.op_linear(0, a_d[:1], w["layers"][0]["w_qkv"], None, o_qkv[:1])      # synchronising call: surfaces a device-side status
+    dec.op_linear(0, a_d[:1], dec.layer_weights[0]["w_qkv"], None, o_qkv[:1])      # synchronising call: surfaces a device-side status
     ms = ev0.elapsed_time(ev1) / reps
     wbytes = sh.n_layers * 2.0 * ((qd + 2 * kvd) * d + d * qd + 2 * f * d + d * f)
     abytes = sh.n_layers * 2.0 * M * (d + (qd + 2 * kvd) + qd + d + d + f + f + d)

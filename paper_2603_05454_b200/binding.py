@@ -179,6 +179,11 @@ class LSPDecoder:
         except Exception:
             pass
 
+    @property
+    def layer_weights(self):
+        """Per-layer weight tensors as the library holds them (w_qkv is the packed [q; k; v] projection)."""
+        return self._layers
+
     def set_sched(self, sched: SchedCfg):
         self.sched = sched
         sc = sched.to_c()
