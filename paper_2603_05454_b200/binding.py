@@ -195,11 +195,14 @@ class LSPDecoder:
     # -- Algorithm 1
     def begin(self, tokens: torch.Tensor, prompt_len, gen_len):
         assert tokens.dtype == torch.int32 and tokens.is_cuda and tokens.dim() == 2 and tokens.is_contiguous()
-        self.tokens = tokens
-        self.batch = tokens.shape[0]
+        batch = tokens.shape[0]
         pl = np.ascontiguousarray(prompt_len, dtype=np.int32)
         gl = np.ascontiguousarray(gen_len, dtype=np.int32)
-        self._check(lib.lsp_begin(self._h, tokens.data_ptr(), tokens.shape[1], pl.ctypes.data, gl.ctypes.data, self.batch))
+        if pl.shape != (batch,) or gl.shape != (batch,):
+            raise ValueError(f"prompt_len and gen_len need one entry per row of tokens ({batch})")
+        self._check(lib.lsp_begin(self._h, tokens.data_ptr(), tokens.shape[1], pl.ctypes.data, gl.ctypes.data, batch))
+        self.tokens = tokens          # the library state changed only now (a rejected call leaves the old decode in place)
+        self.batch = batch
 
     def denoise_step(self):
         recs = (StepRec * self.batch)()
@@ -211,6 +214,8 @@ class LSPDecoder:
             self._check(lib.lsp_commit(self._h, None))
         else:
             a = np.ascontiguousarray(L, dtype=np.int32)
+            if a.shape != (self.batch,):
+                raise ValueError(f"L needs one entry per sequence ({self.batch})")
             self._check(lib.lsp_commit(self._h, a.ctypes.data))
 
     def generate(self, max_recs: int = 0):
@@ -227,10 +232,13 @@ class LSPDecoder:
         assert tokens_dev.dtype == torch.int32 and tokens_dev.is_cuda and tokens_dev.is_contiguous()
         for t in (tokens_in, tokens_out):
             assert t.dtype == torch.int32 and not t.is_cuda and t.is_contiguous() and t.shape == tokens_dev.shape
-        self.tokens = tokens_dev
-        self.batch = tokens_dev.shape[0]
+        batch = tokens_dev.shape[0]
         pl = np.ascontiguousarray(prompt_len, dtype=np.int32)
         gl = np.ascontiguousarray(gen_len, dtype=np.int32)
+        if pl.shape != (batch,) or gl.shape != (batch,):
+            raise ValueError(f"prompt_len and gen_len need one entry per row of tokens ({batch})")
+        self.tokens = tokens_dev
+        self.batch = batch
         n = C.c_int(0)
         recs = (StepRec * max_recs)() if max_recs else None
         self._check(lib.lsp_generate_host(self._h, tokens_dev.data_ptr(), tokens_dev.shape[1], tokens_in.data_ptr(),

@@ -181,3 +181,37 @@ def test_bf16_tcgen05_attention_head_dim_128(hq, hkv):
     sh = S.ModelShape(2, 128 * hq, hq, hkv, 128, 512, 2048, dtype="bf16", head_scale=1.5, w_std=0.5 / (128 * hq) ** 0.5)
     _teacher_forced(sh, 11, 150, 170, SchedCfg(mode=2, fixed_k=45), (1, 200), attn_impl=2, max_steps=4)
     _teacher_forced(sh, 12, 40, 90, SchedCfg(tau=0.04), (1, 400), attn_impl=2, max_steps=6)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_degenerate_lengths_and_policies(dtype):
+    """The smallest problems the method has (one prompt token, one masked position: a single denoiser pass that runs to
+    the end), a decode that exactly fills max_len, a snapping window of 0 (only the run's own last token can snap), and
+    an L_min larger than the whole suffix (clamped to N)."""
+    from paper_2603_05454_b200 import SchedCfg
+    sh = S.ModelShape(2, 256, 4, 2, 64, 512, 1024, dtype=dtype, head_scale=1.5, w_std=0.0625)
+    n, _ = _teacher_forced(sh, 31, 1, 1, SchedCfg(tau=0.05), (1, 200))
+    assert n == 1
+    _teacher_forced(sh, 32, 1, 33, SchedCfg(tau=0.05), (1, 200))
+    _teacher_forced(sh, 33, 31, 2, SchedCfg(tau=2.0), (1, 200))                  # nothing passes: L <- 1 every step
+    _teacher_forced(sh, 34, 9, 40, SchedCfg(tau=0.05, snap_window=0), (1, 200))
+    _teacher_forced(sh, 35, 9, 24, SchedCfg(tau=0.05, l_min=1000), (1, 200))
+    _teacher_forced(sh, 36, 9, 40, SchedCfg(tau=0.0), (1, 200))                  # everything passes: one pass
+
+
+def test_begin_rejects_empty_and_oversize_sequences():
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg, LSPError
+    sh = S.ModelShape(1, 64, 1, 1, 64, 64, 256, dtype="fp32")
+    dec = LSPDecoder(sh, S.make_weights(sh, 0, device=DEV), SchedCfg(), 2, 16, device=DEV)
+    tokens = torch.zeros(2, 16, dtype=torch.int32, device=DEV)
+    for P, G in (([0, 4], [4, 4]), ([4, 4], [0, 4]), ([4, 9], [4, 8]), ([4, 4], [4, -1])):
+        with pytest.raises(LSPError):
+            dec.begin(tokens, P, G)
+    with pytest.raises(ValueError):
+        dec.begin(tokens, [4, 4, 4], [4, 4, 4])                                  # lengths must match the token rows
+    with pytest.raises(LSPError):
+        dec.begin(torch.zeros(3, 16, dtype=torch.int32, device=DEV), [4, 4, 4], [4, 4, 4])   # more sequences than max_batch
+    dec.begin(tokens, [8, 1], [8, 15])                                           # exactly max_len is fine
+    n, _ = dec.generate()
+    assert n >= 1 and dec.active()[1] == 0
+    dec.close()
