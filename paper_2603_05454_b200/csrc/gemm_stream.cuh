@@ -104,7 +104,8 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   constexpr int ACC = (MT == 1 && NI == 2) ? 2 : 1;       // accumulators per row tile
   constexpr int SET_COLS = MT * ACC * BN;                 // columns of one accumulator set
   constexpr int NBUF = (2 * SET_COLS <= 512) ? 2 : 1;     // accumulator sets in tensor memory
-  constexpr uint32_t TMEM_COLS = NBUF * SET_COLS;
+  // tensor memory is allocated in powers of two (192-wide tiles use 384 of 512 columns)
+  constexpr uint32_t TMEM_COLS = (NBUF * SET_COLS <= 128) ? 128 : (NBUF * SET_COLS <= 256 ? 256 : 512);
   const int A_ATOM = args.a_rows * 128;
   const int AT = args.atoms;
   const int STAGE_BYTES = AT * (A_ATOM + B_ATOM);
@@ -350,13 +351,15 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             tc_wait_ld();
             tc_pin16(p0);
             if (Epi::kDual) tc_pin16(p1);
-            request(c + 16, q0, q1);
+            if (c + 16 < CH) request(c + 16, q0, q1);
             consume(c, p0, p1);
-            tc_wait_ld();
-            tc_pin16(q0);
-            if (Epi::kDual) tc_pin16(q1);
-            if (c + 32 < CH) request(c + 32, p0, p1);
-            consume(c + 16, q0, q1);
+            if (c + 16 < CH) {                     // CH is a multiple of 16, not always of 32 (48 pairs per tile)
+              tc_wait_ld();
+              tc_pin16(q0);
+              if (Epi::kDual) tc_pin16(q1);
+              if (c + 32 < CH) request(c + 32, p0, p1);
+              consume(c + 16, q0, q1);
+            }
           }
           if constexpr (Epi::kReduce) {
             if (m < args.M) epi.part[(size_t)m * epi.n_tiles + tile] = red;

@@ -513,6 +513,7 @@ struct UmmaState {
                                    // 0 = leave those to the tiled kernel
   int stream_bn = 0;               // its tile width with one row tile (0 = automatic)
   int stream_bn2 = 0;              // ... and with two row tiles
+  int stream_bn_dual = 0;          // tile width of dual epilogues: 0 = automatic, 192 or 256
   int stream_atoms = 0;            // K atoms per stage: 0 = two when stream_min_stages2 such stages fit, else 1 or 2 as given
   int stream_min_stages2 = 3;
   int stream_grid_mode = 2;        // its grid: 0 = by row count, 1 = one CTA per SM (even shares), 2 = multiple of the tile count
@@ -625,6 +626,11 @@ int stream_dispatch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf1
   LSP_STREAM_CASE(256, 1, 1);
   LSP_STREAM_CASE(256, 1, 2);
   LSP_STREAM_CASE(256, 2, 2);
+  if constexpr (Epi::kDual && !std::is_same<Epi, EpiQKVRope<bf16>>::value) {    // 96 pairs per tile: whole tiles only (see umma_gemm)
+    if (bn == 192 && mt == 1) ni = 1;
+    LSP_STREAM_CASE(192, 1, 1);
+    LSP_STREAM_CASE(192, 2, 2);
+  }
   if constexpr (!Epi::kReduce) {
     LSP_STREAM_CASE(128, 1, 1);
     LSP_STREAM_CASE(128, 1, 2);
@@ -687,8 +693,23 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
       if (M <= UM_BM && st.stream_bn > 0) sbn = st.stream_bn;
       if (M > UM_BM && M <= 2 * UM_BM && st.stream_bn2 > 0) sbn = st.stream_bn2;
       if (box_rows > sbn / 2) sbn = 2 * box_rows;
+      if constexpr (Epi::kDual && !std::is_same<Epi, EpiQKVRope<bf16>>::value) {
+        // 192-wide tiles (96 pairs): with 12288 pairs that is 128 tiles instead of 96, i.e. a third more SMs pulling
+        // operands, and a quarter less shared-memory fill per CTA.  Only where no tile would be split between CTAs
+        // (the split paths assume a power-of-two chunk count): one wave of whole tiles, or several row groups.
+        // (The same idea for the rotary QKV GEMM, 96-wide tiles that straddle heads, needs 16-row TMA boxes of 2 KB,
+        // and those cost far more than the fuller wave gains: +0.7 ms per LLaDA-shaped pass.  Not kept.)
+        if (st.stream_bn_dual != 256 && NP % 96 == 0 && st.stream_grid_mode == 2 && st.target_ctas == 0) {
+          const int mt192 = M <= UM_BM ? 1 : 2;
+          const long groups = (M + UM_BM * mt192 - 1) / (UM_BM * mt192);
+          const long t192 = (long)(NP / 96) * groups, t256 = (long)((NP + 127) / 128) * groups;
+          const bool whole192 = (groups == 1 && t192 <= st.n_sm && 2 * t192 > st.n_sm) || (groups > 1 && t192 >= st.n_sm);
+          const bool better = M <= 2 * UM_BM ? (t256 < t192 && t256 < st.n_sm) : false;
+          if (whole192 && (st.stream_bn_dual == 192 || better)) sbn = 192;
+        }
+      }
       const int smt = stream_row_tiles<Epi>(st, M, NP, K, sbn);
-      if (smt > 0 && (sbn == 128 || sbn == 256))
+      if (smt > 0 && (sbn == 128 || sbn == 256 || sbn == 192))
         return stream_dispatch<Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows, sbn, smt,
                                     st.stream_issuers);
     }
