@@ -593,16 +593,16 @@ inline size_t stream_scratch_bytes(int n_ctas, int bn, int mt) { return (size_t)
 // With at most as many tiles as SMs, a grid that is a multiple of the tile count splits each tile into equal K slices
 // instead (no split at all when there are more than half as many tiles as SMs).  Measured on the LLaDA layer shapes
 // the second choice is as fast or faster at every row count from 2 to 128, so it is the default.
-// K slices per tile when the tiles are fewer than the SMs.  With clusters on: a power of two up to 8 (a cluster of 3
-// measured 40 % slower than the same split without clusters), and no more clusters than can be resident at once
-// (sixteen clusters of 8 do not fit the 148 SMs' GPC layout: the launch would run in two waves).
+// K slices per tile when the tiles are fewer than the SMs.  With clusters on, the slices of a tile form one cluster of 2
+// to 8 CTAs, and a launch never asks for more clusters than can be resident at once: the GPC layout fits 74 / 45 / 33 /
+// 26 / 22 / 15 / 15 clusters of 2 ... 8 one-per-SM CTAs, so e.g. 48 clusters of 3 or 16 of 8 would run as two waves
+// (measured: 40 % and 100 % slower than the next smaller split).
 inline int stream_splits(const UmmaState& st, long n_tiles) {
   int splits = n_tiles <= st.n_sm ? (int)(st.n_sm / n_tiles) : 0;
   if (st.stream_cluster && splits > 1) {
-    int p2 = 1, lg = 0;
-    while (2 * p2 <= splits && 2 * p2 <= 8) { p2 *= 2; ++lg; }
-    while (p2 > 1 && n_tiles > st.max_clusters[lg]) { p2 /= 2; --lg; }
-    splits = p2;
+    int c = splits < 8 ? splits : 8;
+    while (c > 1 && n_tiles > st.max_clusters[c]) --c;
+    splits = c;
   }
   return splits;
 }
@@ -642,25 +642,25 @@ inline StreamShape stream_shape(const UmmaState& st, int a_rows, int bn, int mt,
 // Activation box rows: all rows (rounded up to 8) when they fit one group of 128 mt rows, else a full group.
 inline int stream_a_rows(int M, int mt) { return M <= UM_BM * mt ? (M + 7) / 8 * 8 : UM_BM * mt; }
 
-// Asks the runtime how many clusters of 2, 4 and 8 CTAs of the streaming kernel (one CTA per SM) can be resident at once.
+// Asks the runtime how many clusters of 2 ... 8 CTAs of the streaming kernel (one CTA per SM) can be resident at once.
 inline void stream_query_clusters(UmmaState& st) {
   auto kern = k_gemm_stream<128, 1, 1, EpiStore<bf16>>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, st.max_smem) != cudaSuccess) return;
-  st.max_clusters[0] = st.n_sm;
-  for (int lg = 1; lg <= 3; ++lg) {
+  st.max_clusters[1] = st.n_sm;
+  for (int c = 2; c <= 8; ++c) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(8 * st.n_sm);
+    cfg.gridDim = dim3(2 * c * st.n_sm);
     cfg.blockDim = dim3(ST_THREADS);
     cfg.dynamicSmemBytes = (size_t)st.max_smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1u << lg;
+    attr[0].val.clusterDim.x = (unsigned)c;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0) st.max_clusters[lg] = n;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) == cudaSuccess && n > 0) st.max_clusters[c] = n;
   }
   cudaGetLastError();
 }
@@ -696,9 +696,8 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
   int cluster = 0, cl_rounds = 1;
   if (!whole && !Epi::kReduce && st.stream_cluster && grid % T == 0) {
     const int splits = (int)(grid / T);
-    // sizes 2, 4 and 8 only: a cluster of 3 measured 40 % slower than the same split without clusters
     const size_t area = (size_t)sh.stages * sh.stage_bytes, tile_bytes = (size_t)UM_BM * BN * sizeof(float);
-    if ((splits == 2 || splits == 4 || splits == 8) && kc >= splits && area >= tile_bytes) {
+    if (splits >= 2 && splits <= 8 && kc >= splits && area >= tile_bytes) {
       cluster = splits;
       if (area < MT * tile_bytes) cl_rounds = MT;      // the partial tile is published one row tile at a time
     }

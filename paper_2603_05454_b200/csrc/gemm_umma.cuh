@@ -504,7 +504,7 @@ struct UmmaState {
   int skinny_bn = 128;             // tile width of plain epilogues in that regime
   int pdl = 1;                     // launch with the programmatic-serialisation attribute
   int stream_cluster = 1;          // persistent kernel: K slices of a tile on one thread block cluster, reduced through DSMEM
-  int max_clusters[4] = {148, 66, 33, 14};   // clusters of 1, 2, 4, 8 one-per-SM CTAs that can be resident at once (queried at init)
+  int max_clusters[9] = {0, 148, 74, 45, 33, 26, 22, 15, 15};   // [c]: clusters of c one-per-SM CTAs that can be resident at once (queried at init)
   int stream_half_sm = 1;          // persistent kernel: cap shared memory at half an SM when three stages still fit
   int use_stream = 1;              // M <= 128: use the persistent weight-streaming kernel (gemm_stream.cuh)
   int stream_issuers = 1;          // MMA-issuing warps with one row tile per CTA (two row tiles always use two); measured: no gain from 2

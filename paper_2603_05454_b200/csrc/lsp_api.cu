@@ -395,7 +395,8 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
               if (c->N[b] > 0) max_keys = std::max(max_keys, c->F[b] + c->pend[b] + (scattered ? c->G[b] : c->N[b]));
             const int key_tiles = (max_keys + AU_BN - 1) / AU_BN;
             const int ctas = row_tiles * m.n_kv_heads * B;
-            while (cl < 8 && 2 * cl * ctas <= c->umma.n_sm && 2 * cl <= key_tiles) cl *= 2;
+            // ... as long as that many clusters can be resident at once (this kernel, too, runs one CTA per SM)
+            while (cl < 8 && 2 * cl * ctas <= c->umma.n_sm && 2 * cl <= key_tiles && ctas <= c->umma.max_clusters[2 * cl]) cl *= 2;
           }
           dim3 g3(row_tiles * cl, m.n_kv_heads, B);
           const float sl2 = scale * 1.4426950408889634f;
