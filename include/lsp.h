@@ -152,7 +152,9 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * 28 = see key 1, 30 = the tcgen05 attention splits a row tile's keys over a thread block cluster when there are few CTAs
  * (1, default), 29 = the K slices of a split tile run as one thread block cluster and are reduced through distributed
  * shared memory (1, default) or through global scratch by the last CTA to arrive (0), 32 = tile width of the dual
- * (SwiGLU) GEMM in the persistent kernel: 0 = automatic (default), 192 or 256. */
+ * (SwiGLU) GEMM in the persistent kernel: 0 = automatic (default), 192 or 256, 33 = a cluster of 2 exchanges half tiles
+ * (1, default: each CTA keeps the half it finishes in tensor memory) or publishes whole partial tiles like larger
+ * clusters (0). */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

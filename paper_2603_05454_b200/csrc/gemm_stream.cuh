@@ -41,7 +41,8 @@ struct StreamArgs {
   int cluster;      // > 1: the launch uses thread block clusters of this size, one cluster per tile, CTA rank r owning the
                     // r-th K slice; the partial tiles are then reduced through distributed shared memory (see the kernel)
   int cl_rounds;    // ... in this many rounds: 1 = the whole partial tile at once, MT = one row tile (128 rows) at a time,
-                    // for partial tiles larger than the pipeline's shared memory
+                    // for partial tiles larger than the pipeline's shared memory; 0 = clusters of 2 exchange halves (each
+                    // CTA publishes only the half its peer finishes and keeps its own half in tensor memory)
   int kc;           // K chunks (one per stage) per tile
   int a_rows;       // activation box rows (M rounded up to a multiple of 8)
   int atoms;        // 64-element K atoms per stage (1 or 2)
@@ -374,6 +375,37 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         // rows) write and read consecutive 16-byte pieces.
         // With clusters the partial tile goes to this CTA's own shared memory (the pipeline stages are idle by now) and
         // is reduced after the role loops; without, to the global scratch slot of this CTA.
+        if (args.cluster == 2 && args.cl_rounds == 0) {
+          // Exchange between the two CTAs of a pair: each finishes half of the tile's 16-column chunks, so each
+          // publishes only the half its peer will finish and keeps its own half in tensor memory (see below).
+          if constexpr (ACC == 1) {
+            constexpr int P = Epi::kDual ? 2 : 1;
+            const int rank = (int)cluster_ctarank();
+            const int p_lo = (CH / 16) * (1 - rank) / 2, p_hi = (CH / 16) * (2 - rank) / 2;     // the peer's chunks
+            float4* slot = reinterpret_cast<float4*>(smem);
+#pragma unroll 1
+            for (int mt = 0; mt < MT; ++mt) {
+              const int m = mt * UM_BM + r_in;
+#pragma unroll 1
+              for (int ch = p_lo; ch < p_hi; ++ch) {
+#pragma unroll
+                for (int p = 0; p < P; ++p) {
+                  float v[16];
+                  tc_ld16(t_row + mt * BN + p * HALF + ch * 16, v);
+                  if (row0 + m < args.M) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                      slot[(size_t)(((ch - p_lo) * P + p) * 4 + i) * ROWS + m] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                  }
+                }
+              }
+            }
+          }
+          cl_tile = tile;
+          cl_row0 = row0;
+          u = seg_end;
+          continue;
+        }
         float4* slot_base = args.cluster > 1
                                 ? reinterpret_cast<float4*>(smem)
                                 : reinterpret_cast<float4*>(args.scratch + (size_t)(g * 2 + (seg == 0 ? 0 : 1)) * ROWS * BN);
@@ -494,7 +526,53 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
       u = seg_end;
     }
   }
-  if (args.cluster > 1) {
+  if (args.cluster == 2 && args.cl_rounds == 0) {
+    // Pair exchange: after the barrier each CTA adds, for its own half of the chunks, its accumulator (still in tensor
+    // memory) and the peer's published piece, and runs the fused epilogue.  One row per thread, as in the plain epilogue.
+    cluster_sync();
+    if constexpr (!Epi::kReduce && ACC == 1) {
+      if (warp >= 2 && warp <= 5 && n_units > 0) {
+        constexpr int CH = Epi::kDual ? HALF : BN;
+        constexpr int P = Epi::kDual ? 2 : 1;
+        const int rank = (int)cluster_ctarank();
+        const int o_lo = (CH / 16) * rank / 2, o_hi = (CH / 16) * (rank + 1) / 2;               // this CTA's chunks
+        const int q = warp & 3, r_in = q * 32 + lane;
+        const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t peer = cluster_map(smem_u32(smem), (unsigned)(rank ^ 1));
+        const int j0 = cl_tile * CH;
+        tc_fence_after();
+#pragma unroll 1
+        for (int mt = 0; mt < MT; ++mt) {
+          const int m = mt * UM_BM + r_in;
+          const bool live = cl_row0 + m < args.M;
+#pragma unroll 1
+          for (int ch = o_lo; ch < o_hi; ++ch) {
+            float a0[16], a1[16];
+            tc_ld16(t_row + mt * BN + ch * 16, a0);
+            if (Epi::kDual) tc_ld16(t_row + mt * BN + HALF + ch * 16, a1);
+            if (live) {
+              float4 t0[4], t1[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) t0[i] = ld_cluster_f4(peer + (uint32_t)(((((ch - o_lo) * P) * 4 + i) * ROWS + m) * 16));
+              if (Epi::kDual) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) t1[i] = ld_cluster_f4(peer + (uint32_t)(((((ch - o_lo) * P + 1) * 4 + i) * ROWS + m) * 16));
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                a0[4 * i] += t0[i].x; a0[4 * i + 1] += t0[i].y; a0[4 * i + 2] += t0[i].z; a0[4 * i + 3] += t0[i].w;
+                if (Epi::kDual) {
+                  a1[4 * i] += t1[i].x; a1[4 * i + 1] += t1[i].y; a1[4 * i + 2] += t1[i].z; a1[4 * i + 3] += t1[i].w;
+                }
+              }
+              if (j0 + ch * 16 < args.n_pairs) epi16(epi, cl_row0 + m, j0 + ch * 16, a0, a1);
+            }
+          }
+        }
+      }
+    }
+    cluster_sync();      // nobody leaves while its peer may still read its shared memory
+  } else if (args.cluster > 1) {
     // Split-K reduction inside the cluster: every CTA's partial tile sits in its shared memory; after the barrier CTA
     // rank r sums, for its share of the 16-column chunks, the partials of all ranks in rank order (= K order, so the
     // result does not depend on timing) straight from their shared memory, and runs the fused epilogue on them.
@@ -700,6 +778,7 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
     if (splits >= 2 && splits <= 8 && kc >= splits && area >= tile_bytes) {
       cluster = splits;
       if (area < MT * tile_bytes) cl_rounds = MT;      // the partial tile is published one row tile at a time
+      if (splits == 2 && st.stream_exchange && !(MT == 1 && NI == 2) && 2 * area >= MT * tile_bytes) cl_rounds = 0;
     }
   }
   StreamArgs args{M, NP, n_tiles, row_groups, whole, cluster, cl_rounds, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch,

@@ -514,6 +514,7 @@ struct UmmaState {
   int stream_bn = 0;               // its tile width with one row tile (0 = automatic)
   int stream_bn2 = 0;              // ... and with two row tiles
   int stream_bn_dual = 0;          // tile width of dual epilogues: 0 = automatic, 192 or 256
+  int stream_exchange = 1;         // clusters of 2 exchange half tiles instead of publishing whole partial tiles
   int stream_atoms = 0;            // K atoms per stage: 0 = two when stream_min_stages2 such stages fit, else 1 or 2 as given
   int stream_min_stages2 = 3;
   int stream_grid_mode = 2;        // its grid: 0 = by row count, 1 = one CTA per SM (even shares), 2 = multiple of the tile count
@@ -684,10 +685,14 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
       // pairs); plain ones take 128, which needs no K split with 96 tiles, except that a wide GEMM with at most 32
       // rows takes 256 (its partial tiles are small, and half as many MMA instructions are issued).  The rotary
       // epilogue's half tiles are fetched head by head.
-      int sbn = Epi::kDual ? 256 : ((M <= 32 && cols >= 8192) ? 256 : 128), box_rows = 0;
+      // With 129..256 rows (two row tiles per CTA) a wide GEMM again takes 256 columns, its K halves on a cluster of 2
+      // that exchanges half tiles: 256 x 256 tiles need a third less shared-memory fill than 256 x 128 ones (QKV-sized
+      // GEMM 38-40 -> 35-37.5 us); a narrow GEMM (36 tiles of 128) is better off with more, smaller tiles.
+      const bool wide_two_tiles = M > UM_BM && M <= 2 * UM_BM && cols >= 8192 && st.stream_exchange && st.stream_cluster;
+      int sbn = Epi::kDual ? 256 : (((M <= 32 || wide_two_tiles) && cols >= 8192) ? 256 : 128), box_rows = 0;
       if constexpr (std::is_same<Epi, EpiQKVRope<bf16>>::value) {
         box_rows = epi.half;
-        sbn = (M <= 32) ? 256 : 128;
+        sbn = (M <= 32 || wide_two_tiles) ? 256 : 128;
       }
       if (M > 2 * UM_BM || (M > UM_BM && st.stream_two_tiles == 2)) sbn = 256;   // several row groups: the widest MMA
       if (M <= UM_BM && st.stream_bn > 0) sbn = st.stream_bn;

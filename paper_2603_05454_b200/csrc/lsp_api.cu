@@ -702,6 +702,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   else if (key == 27) c->umma.stream_half_sm = value ? 1 : 0;
   else if (key == 29) c->umma.stream_cluster = value ? 1 : 0;
   else if (key == 32) c->umma.stream_bn_dual = (value == 192 || value == 256) ? value : 0;
+  else if (key == 33) c->umma.stream_exchange = value ? 1 : 0;
   else if (key == 26) c->umma.stream_issuers = value == 1 ? 1 : 2;
   else if (key == 24) c->umma.stream_big_mt = (value >= 1 && value <= 3) ? value : 0;
   else if (key == 20) c->umma.stream_bn2 = (value == 256 || value == 128 || value == 64) ? value : 0;

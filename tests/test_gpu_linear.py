@@ -98,6 +98,7 @@ def test_linear_bf16_weight_streaming_kernel(grid_mode, shape):
     (200, 4096, 4096, {20: 256}), (256, 12288, 4096, {20: 256}), (130, 4096, 12288, {20: 256}),
     (640, 4096, 12288, {}), (1000, 3584, 3584, {}), (300, 2048, 1024, {}), (257, 512, 2048, {}),
     (640, 4096, 4096, {29: 0}),
+    (640, 4096, 12288, {33: 0}), (200, 12288, 1024, {20: 256, 33: 0}),      # clusters of 2 without the half-tile exchange
     # SwiGLU GEMM with 192-wide tiles (96 pairs): one and two row tiles, several row groups, a forced 256 for contrast
     (100, 12288, 256, {}), (200, 12288, 320, {}), (600, 12288, 256, {32: 192}), (100, 12288, 256, {32: 256}),
     (300, 9600, 192, {32: 192}),
