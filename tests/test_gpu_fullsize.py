@@ -126,60 +126,81 @@ def test_adaptive_threshold_decode_shrinks_the_suffix_geometrically_at_full_voca
     assert n == max(len([r for r in recs[b::B] if r["n_before"] > 0]) for b in range(B))
 
 
-def test_cfg3_full_depth_decode_in_the_benchmark_configuration_keeps_its_invariants():
-    """The LLaDA-8B-shaped decode exactly as the benchmark runs it (32 layers, full vocabulary, batch 1, 256 + 256,
-    tau 0.9, delimiters 1..32, default kernels), checked against what Algorithm 1 fixes at any size: every step's
-    record is the scan of that step's own scores (run = leading positions with p_max >= tau; block = run or the last
-    delimiter at most W before its end; never 0), the committed tokens are that step's argmaxes, the frozen prefix
-    never changes, the masked suffix shrinks by exactly the committed block, and the KV cache holds exactly the
-    committed prefix minus the block still pending."""
+@pytest.mark.parametrize("name,checked_steps", [("cfg3", 12), ("cfg4", 6)])
+def test_full_depth_decode_in_the_benchmark_configuration_keeps_its_invariants(name, checked_steps):
+    """The LLaDA-8B-shaped decode (cfg3: 32 layers, batch 1, 256 + 256, tau 0.9) and the Dream-7B-shaped one (cfg4: 28
+    layers, grouped-query attention 28/4, batch 4, 512 + 512, tau 0.85) exactly as the benchmark runs them (full
+    vocabulary, default kernels), checked against what Algorithm 1 fixes at any size: every step's record is the scan of
+    that step's own scores (run = leading positions with p_max >= tau; block = run or the last delimiter at most W
+    before its end; never 0), the committed tokens are that step's argmaxes, the frozen prefix never changes, the masked
+    suffix shrinks by exactly the committed block, and the KV cache holds exactly the committed prefix minus the block
+    still pending."""
     from paper_2603_05454_b200 import LSPDecoder, SchedCfg
-    wl = S.config("cfg3")
+    wl = S.config(name)
     sh = wl.shape
     W = 16
     w = S.make_weights(sh, 0, device=DEV)
     bm = S.delimiter_bitmap(sh.vocab, *wl.delim).to(DEV)
-    P, G = wl.prompt_len, wl.gen_len
-    dec = LSPDecoder(sh, w, SchedCfg(tau=wl.tau, snap_window=W, delim_bitmap=bm), 1, P + G, device=DEV)
-    tokens = torch.full((1, P + G), sh.mask_id, dtype=torch.int32, device=DEV)
-    tokens[0, :P] = S.make_prompt(1, P, sh, 100)[0].to(DEV)
-    dec.begin(tokens, [P], [G])
+    B, P, G = wl.batch, wl.prompt_len, wl.gen_len
+    dec = LSPDecoder(sh, w, SchedCfg(tau=wl.tau, snap_window=W, delim_bitmap=bm), B, P + G, device=DEV)
+    tokens = torch.full((B, P + G), sh.mask_id, dtype=torch.int32, device=DEV)
+    tokens[:, :P] = S.make_prompt(B, P, sh, 100).to(DEV)
+    dec.begin(tokens, [P] * B, [G] * B)
     tau32 = np.float32(wl.tau)
-    N, F, pend, frozen = G, 0, P, tokens[0, :P].cpu().numpy().copy()
+    N, F, pend = [G] * B, [0] * B, [P] * B
+    frozen = [tokens[b, :P].cpu().numpy().copy() for b in range(B)]
     steps = 0
-    while N > 0:
-        rec = dec.denoise_step()[0]
-        y, p, m = dec.scores()
-        assert rec["n_before"] == N and rec["rows"] == pend + N and len(p) == N
-        assert (p > 0).all() and (p <= 1.0 + 1e-6).all() and (m >= 0).all() and (y >= 0).all() and (y != sh.mask_id).all()
-        run = int(np.argmax(p < tau32)) if (p < tau32).any() else N
-        assert rec["L_run"] == run
-        if run == N:
-            want = N
-        else:
-            lo = max(1, run - W)
-            delims = [j for j in range(lo, run + 1) if wl.delim[0] <= y[j - 1] <= wl.delim[1]]
-            want = max(1, delims[-1] if delims else run)
-        assert rec["L_commit"] == min(N, max(1, want)), (steps, rec, run)
+    while max(N) > 0 and steps < checked_steps:
+        recs = dec.denoise_step()
+        y_all, p_all, m_all = dec.scores()
+        assert len(p_all) == sum(N)
+        assert (p_all > 0).all() and (p_all <= 1.0 + 1e-6).all() and (m_all >= 0).all()
+        assert (y_all >= 0).all() and (y_all != sh.mask_id).all()
+        off = 0
+        blocks = []
+        for b in range(B):
+            rec = recs[b]
+            if N[b] == 0:
+                assert rec["n_before"] == 0
+                blocks.append(None)
+                continue
+            y, p = y_all[off:off + N[b]], p_all[off:off + N[b]]
+            off += N[b]
+            assert rec["n_before"] == N[b] and rec["rows"] == pend[b] + N[b]
+            run = int(np.argmax(p < tau32)) if (p < tau32).any() else N[b]
+            assert rec["L_run"] == run
+            if run == N[b]:
+                want = N[b]
+            else:
+                delims = [j for j in range(max(1, run - W), run + 1) if wl.delim[0] <= y[j - 1] <= wl.delim[1]]
+                want = max(1, delims[-1] if delims else run)
+            assert rec["L_commit"] == min(N[b], max(1, want)), (steps, b, rec, run)
+            blocks.append(y[:rec["L_commit"]].copy())
         dec.commit()
-        L = rec["L_commit"]
-        tk = tokens[0].cpu().numpy()
-        assert np.array_equal(tk[:len(frozen)], frozen)                       # prefix immutability
-        assert np.array_equal(tk[len(frozen):len(frozen) + L], y[:L])          # the block is this step's argmaxes
-        assert (tk[len(frozen) + L:] == sh.mask_id).all()
-        frozen = tk[:len(frozen) + L].copy()
-        F, pend, N = F + pend, L, N - L
+        tk = tokens.cpu().numpy()
+        for b in range(B):
+            if blocks[b] is None:
+                continue
+            L, f = len(blocks[b]), len(frozen[b])
+            assert np.array_equal(tk[b, :f], frozen[b])                         # prefix immutability
+            assert np.array_equal(tk[b, f:f + L], blocks[b])                    # the block is this step's argmaxes
+            assert (tk[b, f + L:] == sh.mask_id).all()
+            frozen[b] = tk[b, :f + L].copy()
+            F[b], pend[b], N[b] = F[b] + pend[b], L, N[b] - L
         steps += 1
-        if steps == 12:                                                        # the rest in one call
-            n_more, recs = dec.generate(max_recs=G + 1)
-            live = [r for r in recs if r["n_before"] > 0]
-            assert sum(r["L_commit"] for r in live) == N and all(r["L_commit"] >= 1 for r in live)
-            F, pend, N = F + pend + sum(r["L_commit"] for r in live[:-1]), live[-1]["L_commit"], 0
-            break
+    if max(N) > 0:                                                              # the rest in one call
+        n_more, recs = dec.generate(max_recs=B * (G + 1))
+        for b in range(B):
+            live = [r for r in recs[b::B] if r["n_before"] > 0]
+            assert sum(r["L_commit"] for r in live) == N[b] and all(r["L_commit"] >= 1 for r in live)
+            if live:
+                F[b], pend[b] = F[b] + pend[b] + sum(r["L_commit"] for r in live[:-1]), live[-1]["L_commit"]
+            N[b] = 0
     assert dec.active()[1] == 0 and int((tokens == sh.mask_id).sum()) == 0
-    assert np.array_equal(tokens[0, :len(frozen)].cpu().numpy(), frozen)
     kv = dec.kv_view()
-    assert F + pend == P + G
-    assert bool((kv[:, :, 0, :F].float().abs().amax(dim=(-1, -2)) > 0).all())      # every cached row was written ...
-    assert not bool(kv[:, :, 0, F:].any())                                          # ... and nothing beyond the cache length
+    for b in range(B):
+        assert np.array_equal(tokens[b, :len(frozen[b])].cpu().numpy(), frozen[b])
+        assert F[b] + pend[b] == P + G
+        assert bool((kv[:, :, b, :F[b]].float().abs().amax(dim=(-1, -2)) > 0).all())   # every cached row was written ...
+        assert not bool(kv[:, :, b, F[b]:].any())                                       # ... and nothing beyond the cache length
     dec.close()
