@@ -568,6 +568,12 @@ def main():
     torch.cuda.set_device(dev)
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=dev)
+    if world > 1 and args.workload in ("cfg2", "cfg5"):
+        # single-GPU measurements (the head alone; the topology comparison): rank 0 runs them, the others leave
+        torch.distributed.destroy_process_group()
+        if rank != 0:
+            return 0
+        world = 1
     peaks, peak_kind = load_peaks()
     uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
     sampler = ClockSampler(uuid)
