@@ -133,3 +133,48 @@ def test_linear_bf16_cluster_split_of_two_row_tiles(case):
     ref = g / (1 + np.exp(-g)) * u
     np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05)
     dec.close()
+
+
+def test_linear_bf16_seeded_random_shapes_and_kernel_options():
+    """Sixty seeded random (rows, columns, K, option) combinations across the row regimes (one tile, two tiles, row
+    groups), the split paths (clusters of 2..8, half-tile exchange, rounds, global scratch) and the tile widths."""
+    import random
+    rng = random.Random(7)
+    dec = _dec("bf16")
+    defaults = {29: 1, 33: 1, 20: 0, 23: 0, 32: 0, 17: 2, 24: 3}
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    rows = [1, 2, 5, 17, 32, 33, 64, 100, 128, 129, 190, 256, 257, 300, 400, 512, 640, 768, 1000, 1100, 1536, 2100]
+    done = 0
+    while done < 60:
+        M, N, K = rng.choice(rows), rng.choice([96, 128, 384, 1152, 2048, 3584, 4096, 4608, 9600, 12288]), \
+            rng.choice([64, 192, 320, 1024, 2048, 3584, 4096])
+        if M * N * K > 2e10:
+            continue
+        opts = {}
+        for key, p, vals in ((29, 0.2, [0]), (33, 0.2, [0]), (20, 0.15, [128, 256]), (23, 0.15, [128, 256]),
+                             (32, 0.15, [192, 256]), (17, 0.1, [1]), (24, 0.1, [1, 2])):
+            if rng.random() < p:
+                opts[key] = rng.choice(vals)
+        for k, v in {**defaults, **opts}.items():
+            dec.set_option(k, v)
+        A = S.normal((M, K), done, 1, 1.0, torch.bfloat16, DEV)
+        W = S.normal((N, K), done, 2, 0.05, torch.bfloat16, DEV)
+        W2 = S.normal((N, K), done, 3, 0.05, torch.bfloat16, DEV)
+        X0 = S.normal((M, N), done, 4, 1.0, torch.bfloat16, DEV)
+        a, w, w2, x0 = f64(A), f64(W), f64(W2), f64(X0)
+        rtol = 1.0 / 128
+        out = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+        tag = f"M={M} N={N} K={K} options={opts}"
+        dec.op_linear(0, A, W, None, out)
+        ref = a @ w.T
+        np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05, err_msg=tag)
+        xr = X0.clone()
+        dec.op_linear(1, A, W, None, xr)
+        ref = x0 + a @ w.T
+        np.testing.assert_allclose(f64(xr), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05, err_msg=tag)
+        dec.op_linear(2, A, W, W2, out)
+        g, u = a @ w.T, a @ w2.T
+        ref = g / (1 + np.exp(-g)) * u
+        np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05, err_msg=tag)
+        done += 1
+    dec.close()
