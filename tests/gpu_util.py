@@ -29,6 +29,13 @@ def tol_logit(dtype, z_rms, n_layers=1):
     return max(2e-2, 2.0 ** -8 * 4.5 * (6.0 * max(1, n_layers)) ** 0.5 * z_rms)
 
 
+def tol_prob(dtype, tol_z):
+    """Tolerance on p_max given the logit tolerance tol_z of the same model: p_max = softmax(z)_max, so
+    |dp| = p (1 - p) |dz_max - sum_j w_j dz_j| <= |dz| / 4 with dz the error of the top logit against the softmax-
+    weighted mean of the others' errors (which averages down).  Never below the fixed probability tolerance."""
+    return max(tol_for(dtype), 0.25 * tol_z) if dtype != "fp32" else tol_for(dtype)
+
+
 def make_pair(shape, seed):
     """Weights on the GPU (for the library) and the oracle model built from the CPU copy of the same values."""
     w_gpu = S.make_weights(shape, seed, device=DEV)

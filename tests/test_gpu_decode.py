@@ -7,23 +7,34 @@ import torch
 import lsp_synth as S
 from oracle import scan as oscan
 from oracle.decode import decode, make_is_delim
-from gpu_util import DEV, make_pair, oracle_policy, tol_for, tol_logit
+from gpu_util import tol_prob, DEV, make_pair, oracle_policy, tol_for, tol_logit
 
 pytestmark = pytest.mark.gpu
 NEAR = oscan.FLAG_NEAR_THRESHOLD | oscan.FLAG_NEAR_TIE
 
 
-def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, max_steps=None):
+def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, max_steps=None, gains_seed=None):
     """Runs the GPU path step by step, committing the ORACLE's lengths, and compares every step's outputs."""
     from paper_2603_05454_b200 import LSPDecoder
     tol = tol_for(shape.dtype)
-    w_gpu, om = make_pair(shape, seed)
+    if gains_seed is None:
+        w_gpu, om = make_pair(shape, seed)
+    else:
+        # layer-norm gains that are not all ones (the generator gives the same values on both devices)
+        from oracle import dlm
+        w_gpu, w_cpu = S.make_weights(shape, seed, device=DEV), S.make_weights(shape, seed, device="cpu")
+        for wd, dv in ((w_gpu, DEV), (w_cpu, "cpu")):
+            for l, lw in enumerate(wd["layers"]):
+                for k, name in enumerate(("attn_norm", "ffn_norm")):
+                    lw[name] = (1.0 + S.normal((shape.d_model,), gains_seed, 900 + 2 * l + k, 0.25, torch.float32, dv)).to(lw[name].dtype)
+        om = dlm.OracleDLM(shape, w_cpu)
     prompt = S.make_prompt(1, P, shape, seed)
     sched.delim_bitmap = S.delimiter_bitmap(shape.vocab, *delim).to(DEV)
     zr = []
     decode(om, prompt[0].numpy(), G, make_is_delim(*delim), oracle_policy(sched), max_steps=1,
            on_step=lambda rec, lg, k, v: zr.append(float(np.sqrt((lg * lg).mean()))))
     tol_z = tol_logit(shape.dtype, zr[0], shape.n_layers)
+    tol_p = tol_prob(shape.dtype, tol_z)
     sched.flag_tol = tol_z if sched.score == 1 else tol
     sched.tie_tol = tol_z
     otok, orecs, (ock, ocv) = decode(om, prompt[0].numpy(), G, make_is_delim(*delim), oracle_policy(sched),
@@ -44,7 +55,7 @@ def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, 
         rec = dec.denoise_step()[0]
         y, p, m = dec.scores()
         assert rec["n_before"] == o["n_before"] and rec["rows"] == o["rows"]
-        assert np.abs(p - o["pmax"]).max() <= tol, (o["step"], np.abs(p - o["pmax"]).max())
+        assert np.abs(p - o["pmax"]).max() <= tol_p, (o["step"], np.abs(p - o["pmax"]).max(), tol_p)
         assert np.abs(m - o["delta"]).max() <= tol_z, (o["step"], np.abs(m - o["delta"]).max(), tol_z)
         diff = np.nonzero(y != o["yhat"])[0]
         assert all(o["delta"][i] <= tol_z for i in diff), "argmax differs away from a near-tie"
@@ -215,3 +226,11 @@ def test_begin_rejects_empty_and_oversize_sequences():
     n, _ = dec.generate()
     assert n >= 1 and dec.active()[1] == 0
     dec.close()
+
+
+def test_bf16_model_with_learned_norm_gains():
+    """Layer-norm gains that are not all ones (the synthetic models elsewhere have unit gains)."""
+    from paper_2603_05454_b200 import SchedCfg
+    sh = S.ModelShape(3, 512, 4, 2, 128, 1024, 4096, dtype="bf16", head_scale=1.5, w_std=0.044)
+    _teacher_forced(sh, 41, 40, 90, SchedCfg(tau=0.04), (1, 400), gains_seed=5)
+    _teacher_forced(sh, 42, 200, 140, SchedCfg(mode=2, fixed_k=50), (1, 400), gains_seed=6, max_steps=3)
