@@ -57,7 +57,7 @@ NCU_TRAFFIC = {
     # k_gemm_stream<256,1,1,EpiHead>, 64 rows: profiles/k_gemm_stream_head_M64_V126464.md
     "head": {"captured_bytes": 1062.5e6, "algorithmic_bytes": 1037.0e6, "src": "080274371e48"},
     # k_attn_umma, 16 x (128 query rows over 2048 keys): profiles/k_attn_umma_B16_F1920.md
-    "attn": {"captured_bytes": 569.4e6, "algorithmic_bytes": 570.4e6, "src": "7c526865222c"},
+    "attn": {"captured_bytes": 571.3e6, "algorithmic_bytes": 570.4e6, "src": "fca4873c0292"},
     # k_commit_append of a 16 x 1920-row prompt block: profiles/k_commit_append_prompt_B16_P1920.md
     "commit": {"captured_bytes": 1969.1e6, "algorithmic_bytes": 2013.3e6, "src": "c62d33c71cc9"},
 }

@@ -38,6 +38,12 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const float (&v)[16]) {
         "r"(__float_as_uint(v[15]))
       : "memory");
 }
+// Placed after tc_wait_ld(): makes every later use of v[0..15] depend on a statement that follows the wait, so that the
+// compiler cannot schedule arithmetic on the loaded values ahead of it.
+__device__ __forceinline__ void tc_pin16p(float* v) {
+  asm volatile("" : "+f"(v[0]), "+f"(v[1]), "+f"(v[2]), "+f"(v[3]), "+f"(v[4]), "+f"(v[5]), "+f"(v[6]), "+f"(v[7]), "+f"(v[8]),
+               "+f"(v[9]), "+f"(v[10]), "+f"(v[11]), "+f"(v[12]), "+f"(v[13]), "+f"(v[14]), "+f"(v[15]));
+}
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -238,6 +244,8 @@ k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ 
 #pragma unroll
       for (int c = 0; c < AU_BN; c += 16) tc_ld16_nowait(lane_base + 128u + (uint32_t)(s * AU_BN + c), sv + c);
       tc_wait_ld();
+#pragma unroll
+      for (int c = 0; c < AU_BN; c += 16) tc_pin16p(sv + c);      // no use of the scores may be scheduled ahead of the wait
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(6 + s));          // S buffer read
