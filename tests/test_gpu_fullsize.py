@@ -204,3 +204,27 @@ def test_full_depth_decode_in_the_benchmark_configuration_keeps_its_invariants(n
         assert bool((kv[:, :, b, :F[b]].float().abs().amax(dim=(-1, -2)) > 0).all())   # every cached row was written ...
         assert not bool(kv[:, :, b, F[b]:].any())                                       # ... and nothing beyond the cache length
     dec.close()
+
+
+def test_full_depth_decode_is_reproducible_bit_for_bit():
+    """Every reduction on the path has a fixed order (split-K partials in K order, vocab tiles in tile order, the scan in
+    position order), so repeating a decode must reproduce the tokens and every step record exactly: cfg3 at full depth,
+    in the adaptive-threshold mode (11 passes that cross every row regime from 512 rows down to 2)."""
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+    wl = S.config("cfg3")
+    sh = wl.shape
+    w = S.make_weights(sh, 0, device=DEV)
+    bm = S.delimiter_bitmap(sh.vocab, *wl.delim).to(DEV)
+    P, G = wl.prompt_len, wl.gen_len
+    dec = LSPDecoder(sh, w, SchedCfg(mode=1, alpha=0.25, beta=0.5, delim_bitmap=bm), 1, P + G, device=DEV)
+    prompt = S.make_prompt(1, P, sh, 100).to(DEV)
+    runs = []
+    for _ in range(3):
+        tokens = torch.full((1, P + G), sh.mask_id, dtype=torch.int32, device=DEV)
+        tokens[:, :P] = prompt
+        dec.begin(tokens, [P], [G])
+        n, recs = dec.generate(max_recs=G + 1)
+        runs.append((n, tokens.cpu().numpy().copy(), [(r["L_run"], r["L_commit"], r["flags"], r["tau_used"]) for r in recs]))
+    dec.close()
+    for n, tk, rc in runs[1:]:
+        assert n == runs[0][0] and np.array_equal(tk, runs[0][1]) and rc == runs[0][2]
