@@ -181,7 +181,9 @@ __device__ __forceinline__ void epi16(const EpiResidual<bf16>& e, int m, int j, 
 __device__ __forceinline__ void epi16(const EpiSwiGLU<bf16>& e, int m, int j, const float* g, const float* u) {
   float r[16];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) r[i] = g[i] / (1.f + __expf(-g[i])) * u[i];
+  // __fdividef (reciprocal + multiply, 2 ulp): the IEEE division's slow path is a subroutine call inside the epilogue,
+  // and its mere presence cost the whole kernel 5-7 us at every row count (39.4 -> 34.4 us at 2 rows, 61.7 -> 54.6 at 256)
+  for (int i = 0; i < 16; ++i) r[i] = __fdividef(g[i], 1.f + __expf(-g[i])) * u[i];
   uint4* p = reinterpret_cast<uint4*>(e.out + (size_t)m * e.ld + j);
   p[0] = pack8(r);
   p[1] = pack8(r + 8);
