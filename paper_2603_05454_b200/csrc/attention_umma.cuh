@@ -310,7 +310,7 @@ k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ 
     if (C == 1) {
       if (have) {
         const int row = row_base + r;
-        const float inv = 1.f / l;
+        const float inv = __fdividef(1.f, l);
         const bool valid = row < rows_total;
         const int qi = valid ? row / G : 0, hg = valid ? row % G : 0;
         uint4* dst = reinterpret_cast<uint4*>(out + (size_t)(r0 + qi) * ldq + (kvh * G + hg) * DH);
@@ -366,7 +366,7 @@ k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ 
         wgt[p] = (wgt[p] == -INFINITY) ? 0.f : ex2_approx(wgt[p] - mmax);
         L += wgt[p] * ld_cluster_f1(cluster_map(base_m + 4u * (AU_BM + r), (unsigned)p));
       }
-      const float inv = 1.f / L;
+      const float inv = __fdividef(1.f, L);
       const int qi = valid ? row / G : 0, hg = valid ? row % G : 0;
       uint4* dst = reinterpret_cast<uint4*>(out + (size_t)(r0 + qi) * ldq + (kvh * G + hg) * DH);
       const int ch_lo = (DH / 16) * rank / C, ch_hi = (DH / 16) * (rank + 1) / C;

@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(RN_THREADS) k_rmsnorm(const T* __restrict__ x,
   float tot = 0.f;
 #pragma unroll
   for (int w = 0; w < RN_THREADS / 32; ++w) tot += red[w];      // same order in every thread
-  const float inv = rsqrtf(tot / (float)d + eps);
+  const float inv = rsqrtf(__fdividef(tot, (float)d) + eps);      // fast division: no IEEE slow-path subroutine in the kernel
   if (in_regs) {
 #pragma unroll
     for (int j = 0; j < RN_VPT; ++j) {
@@ -150,7 +150,7 @@ __global__ void k_merge_partials(const Top2* __restrict__ part, int n_tiles, int
   for (int o = 16; o > 0; o >>= 1) t = top2_merge(t, top2_shfl_xor(t, o));
   if (lane == 0) {
     yhat[r] = t.i1;
-    pmax[r] = 1.f / t.s;
+    pmax[r] = __fdividef(1.f, t.s);
     margin[r] = t.m1 - t.m2;
   }
 }
