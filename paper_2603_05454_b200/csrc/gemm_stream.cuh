@@ -79,9 +79,11 @@ __device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
 }
 
 // first unit of CTA g when U units are dealt to G CTAs
-__device__ __forceinline__ long st_first_unit(long U, int G, int g) { return U * g / G; }
+// (units are counted in 32 bits: a 64-bit division is a subroutine call, which no path of this kernel may contain; the
+// host checks that U * G fits)
+__device__ __forceinline__ int st_first_unit(int U, int G, int g) { return (int)((unsigned)U * (unsigned)g / (unsigned)G); }
 // CTA that owns unit u
-__device__ __forceinline__ int st_owner(long U, int G, long u) { return (int)(((u + 1) * G + U - 1) / U) - 1; }
+__device__ __forceinline__ int st_owner(int U, int G, int u) { return (int)(((unsigned)(u + 1) * (unsigned)G + (unsigned)U - 1u) / (unsigned)U) - 1; }
 
 constexpr int ST_THREADS = 224;            // warp 0 producer, warps 1 and 6 MMA issuers, warps 2..5 epilogue
 
@@ -127,13 +129,13 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
 
   const int G = gridDim.x, g = blockIdx.x;
   const int RG = args.row_groups;
-  const long T = (long)args.n_tiles * RG;
-  const long U = T * args.kc;
+  const int T = args.n_tiles * RG;
+  const int U = T * args.kc;
   // Split shares: CTA g owns the contiguous units [U g / G, U (g + 1) / G).  Whole-tile shares: CTA g owns tiles
   // g, g + G, g + 2 G, ... (units are then counted within its own tiles), so that the CTAs running at any moment work
   // on neighbouring tiles: the same few weight tiles for every row group, which keeps the working set inside L2.
-  const long u0 = args.whole_tiles ? 0 : st_first_unit(U, G, g);
-  const long u1 = args.whole_tiles ? ((T - g + G - 1) / G) * args.kc : st_first_unit(U, G, g + 1);
+  const int u0 = args.whole_tiles ? 0 : st_first_unit(U, G, g);
+  const int u1 = args.whole_tiles ? ((T - g + G - 1) / G) * args.kc : st_first_unit(U, G, g + 1);
   const int n_units = (int)(u1 - u0);
   int cl_tile = 0, cl_row0 = 0;      // cluster mode: the tile this CTA contributed a K slice to
 
@@ -210,7 +212,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   if (warp == 0) {
     // ---------------- TMA producer: one uninterrupted stream over this CTA's units ----------------
     if (lane == 0) {
-      long issued = 0;
+      int issued = 0;
       Pos p;
       pos_set(p, (int)(u0 / args.kc), (int)(u0 % args.kc));
       int s = 0;
@@ -232,8 +234,8 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         pos_next(p);
       }
       // do not leave while copies may still be landing in this CTA's shared memory
-      const long first = issued > S ? issued - S : 0;
-      for (long it = first; it < issued; ++it) {
+      const int first = issued > S ? issued - S : 0;
+      for (int it = first; it < issued; ++it) {
         volatile uint32_t no_abort = 0;
         mbar_wait(full_bar((int)(it % S)), (uint32_t)(it / S) & 1u, &no_abort);
       }
@@ -247,9 +249,9 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
       bool ok = true;
       int s = 0;
       uint32_t ph = 0;
-      for (long u = u0; u < u1 && ok;) {
+      for (int u = u0; u < u1 && ok;) {
         const int vt = (int)(u / args.kc);
-        const long seg_end = min(u1, (long)(vt + 1) * args.kc);
+        const int seg_end = min(u1, (vt + 1) * args.kc);
         const int buf = seg % NBUF, use = seg / NBUF;
         // wait until the epilogue has drained this accumulator set (its previous use was segment seg - NBUF)
         if (use >= 1 && !mbar_wait(acce_bar(buf), (uint32_t)(use - 1) & 1u, abort_flag)) {
@@ -295,12 +297,12 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     constexpr int CH = Epi::kDual ? HALF : BN;            // pair indices (dual) or columns (plain) per tile
     int seg = 0;
     bool ok = true;
-    for (long u = u0; u < u1 && ok; ++seg) {
+    for (int u = u0; u < u1 && ok; ++seg) {
       const int vt = (int)(u / args.kc);
       const int tlin = args.whole_tiles ? g + vt * G : vt;
       const int tile = tlin / RG, row0 = (tlin % RG) * ROWS;      // column tile, first activation row
-      const long tile_u0 = (long)vt * args.kc;
-      const long seg_end = min(u1, tile_u0 + args.kc);
+      const int tile_u0 = vt * args.kc;
+      const int seg_end = min(u1, tile_u0 + args.kc);
       const bool whole = (u == tile_u0) && (seg_end == tile_u0 + args.kc);
       const int buf = seg % NBUF, use = seg / NBUF;
       if (!mbar_wait(accf_bar(buf), (uint32_t)use & 1u, abort_flag)) {
@@ -770,6 +772,7 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
   const int whole = (row_groups > 1 && T >= st.n_sm) ? 1 : 0;
   int grid = whole ? st.n_sm : stream_grid(st, (int)T, M);
   if (grid > T * kc) grid = (int)(T * kc);
+  if ((double)T * kc * (grid + 1) >= 4.0e9) { st.err = "too many work units for the streaming GEMM"; return -9; }   // 32-bit unit arithmetic
   // K slices of one tile on the CTAs of one cluster: the reduction then stays on chip
   int cluster = 0, cl_rounds = 1;
   if (!whole && !Epi::kReduce && st.stream_cluster && grid % T == 0) {
