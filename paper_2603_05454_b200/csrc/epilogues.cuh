@@ -103,4 +103,35 @@ struct EpiHead {
   __device__ __forceinline__ bool valid(int j) const { return j < vocab && j != exclude_id; }
 };
 
+// Sixteen consecutive logits z[0..15] of columns col0.. pushed into the running reduction without data-dependent
+// branches: the top-2 state by compare-and-select per element (strict ">" keeps the lowest id on ties, as top2_push),
+// the sum rescaled once per chunk to the new maximum and the sixteen exponentials independent of one another.
+// Equivalent to sixteen top2_push calls up to the rounding of the sum.
+__device__ __forceinline__ void top2_push16(Top2& t, const float* z, int col0, const EpiHead& e) {
+  float v[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = e.valid(col0 + i) ? z[i] : -INFINITY;
+  float cm = v[0];
+#pragma unroll
+  for (int i = 1; i < 16; ++i) cm = fmaxf(cm, v[i]);
+  if (cm == -INFINITY) return;                       // nothing valid in this chunk (uniform per thread, rare)
+  const float m_new = fmaxf(t.m1, cm);
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) sum += __expf(v[i] - m_new);          // exp(-inf) = 0 for the masked columns
+  t.s = t.s * __expf(t.m1 - m_new) + sum;            // t.m1 = -inf on the first chunk: exp(-inf) = 0, t.s = 0
+  float m1 = t.m1, m2 = t.m2;
+  int i1 = t.i1;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const bool gt = v[i] > m1;
+    m2 = gt ? m1 : fmaxf(m2, v[i]);
+    i1 = gt ? col0 + i : i1;
+    m1 = gt ? v[i] : m1;
+  }
+  t.m1 = m1;
+  t.m2 = m2;
+  t.i1 = i1;
+}
+
 }  // namespace lsp

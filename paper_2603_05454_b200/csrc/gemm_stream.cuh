@@ -334,11 +334,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
               }
             }
             if constexpr (Epi::kReduce) {
-#pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const int col = j0 + c + i;
-                if (epi.valid(col)) top2_push(red, a0[i], col);
-              }
+              top2_push16(red, a0, j0 + c, epi);
             } else {
               if (m < args.M && j0 + c < args.n_pairs) epi16(epi, m, j0 + c, a0, a1);
             }
@@ -509,13 +505,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             }
             if constexpr (Epi::kReduce) {
               Top2 red = top2_empty();
-              if (valid) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                  const int col = j0 + c + i;
-                  if (epi.valid(col)) top2_push(red, a0[i], col);
-                }
-              }
+              if (valid) top2_push16(red, a0, j0 + c, epi);
 #pragma unroll
               for (int o = 1; o < NCH; o <<= 1) red = top2_merge(red, top2_shfl_xor(red, o));
               if (valid && ch == 0) epi.part[(size_t)(row0 + mm) * epi.n_tiles + tile] = red;
