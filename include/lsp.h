@@ -220,17 +220,34 @@ int lsp_scan(lsp_ctx* ctx, const float* score, const int32_t* yhat, const float*
 int lsp_op_linear(lsp_ctx* ctx, int op, const void* A, const void* W, const void* W2, void* out, int M,
                   int N, int K);
 
+/* The suffix-over-prefix attention of one layer alone (Sec. 3.2, "bidirectional lookahead" over the frozen prefix and
+ * the active suffix; the attention inside Algorithm 1's forward pass), for parity checks at full head shapes:
+ *   out[r, h, :] = softmax_j(q[r, h, :] . k_j / sqrt(head_dim)) v_j    over j in cache[0, cache_len[b]) then the pass's
+ * own rows of sequence b, no mask; query head h reads KV head h / (n_heads / n_kv_heads).
+ *   q, out        device [rows_total, n_heads * head_dim] T, sequences packed back to back (rows_total = sum rows[b])
+ *   k_new, v_new  device [rows_total, n_kv_heads * head_dim] T: this pass's keys / values (already rotated); they are
+ *                 copied into the context's staging planes of `layer`
+ *   cache_len, rows   host [batch]; the cached keys / values are read from the caller's kv_cache, layer `layer`,
+ *                 sequence slot b, positions [0, cache_len[b]) (layout: lsp_kv_cache_bytes)
+ * Takes the same kernel choice as lsp_denoise_step would for these sizes (lsp_get_counters 16, 17 tell which).
+ * Must not be called between lsp_denoise_step and lsp_commit (it overwrites the step's descriptor: the pending
+ * proposal is dropped).  Synchronises the stream; returns LSP_ERR_DEVICE_TIMEOUT like a step. */
+int lsp_op_attention(lsp_ctx* ctx, int layer, const void* q, const void* k_new, const void* v_new, void* out,
+                     const int32_t* cache_len, const int32_t* rows, int batch);
+
 /* Device time (ms) accumulated since lsp_reset_counters() by kernel class, host float[8]:
  * 0 embed+norms, 1 layer GEMMs, 2 attention, 3 fused LM head, 4 merge+scan, 5 commit/append, 6 whole steps
  * (always filled), 7 host time spent queueing those steps' launches (always filled).  Classes 0-5 are only filled while option key 2 (per-class CUDA-event timing)
  * is 1.  Synchronises the stream. */
 int lsp_last_timing(lsp_ctx* ctx, float* ms);
 
-/* Host-side accounting since lsp_reset_counters(), host double[16]: 0 kernel launches, 1 layer-GEMM algorithmic
+/* Host-side accounting since lsp_reset_counters(), host double[18]: 0 kernel launches, 1 layer-GEMM algorithmic
  * bytes (every operand and result once), 2 layer-GEMM flops, 3 attention bytes (every K/V row once per layer
  * plus Q and O), 4 KV-append bytes (read + write), 5 LM-head bytes, 6 LM-head flops, 7 denoiser passes,
  * 8..13 kernel launches by class (same classes as lsp_last_timing 0..5), 14 attention flops
- * (4 * queries * keys * n_heads * head_dim per layer), 15 committed tokens. */
+ * (4 * queries * keys * n_heads * head_dim per layer), 15 committed tokens; not counters but the last attention
+ * launch: 16 its kernel (0 CUDA cores, 1 mma.sync, 2 tcgen05), 17 the thread block cluster size its key tiles were
+ * split over (1 = no split). */
 int lsp_get_counters(lsp_ctx* ctx, double* out);
 int lsp_reset_counters(lsp_ctx* ctx);
 
@@ -243,7 +260,11 @@ int lsp_reset_counters(lsp_ctx* ctx);
  *   A, W, out  device pointers, 16-byte aligned, row-major, bfloat16; out is written completely.
  *   limits     1 <= M <= 128; N a multiple of 16, at most 524288; K a multiple of 64.  Anything else returns
  *              LSP_ERR_SHAPE (NULL or misaligned pointers: LSP_ERR_ARG) and writes a message into err.
- *   cuda_stream  a cudaStream_t (NULL = default stream); the call only enqueues work and returns.
+ *   cuda_stream  a cudaStream_t (NULL = default stream); the call only enqueues work and returns.  It never reads
+ *              anything back, so a device-side bounded wait that expires inside the kernel (2 s; a protocol fault,
+ *              not a data-dependent event) is NOT reported by this entry point: `out` is then left partly written
+ *              and the call has long since returned LSP_OK.  A caller that must know runs the same product once
+ *              through lsp_op_linear, which synchronises and returns LSP_ERR_DEVICE_TIMEOUT.
  *   err, err_len  optional host buffer that receives a message when the call fails.
  * The first call on a device looks up the array's device address and sets a kernel attribute, once, with that
  * device current; make that first call outside any stream capture.  Every call uses the same array: it clears the

@@ -16,7 +16,7 @@ Readings taken where the paper is silent or inconsistent:
     the L_min fallback to blocks shorter than L_min);
   * finally 1 <= L <= N (Algorithm 1's "if L = 0 then L <- 1").
 
-Pins: exhaustive brute force over all pass/delimiter patterns for N <= 10, tau = 0 and
+Pins: brute force over all pass patterns for N <= 12 (all delimiter patterns for N <= 8), tau = 0 and
 tau = +inf special cases, fixed-k closed form (Table 2), adaptive range invariant and the
 15-step geometric sequence.  The choice of m inside the adaptive range is "parity unpinned"
 (the paper does not state it).

@@ -17,7 +17,7 @@ FLAG_RUN_TO_END, FLAG_NEAR_THRESHOLD, FLAG_NEAR_TIE = 8, 16, 32
 
 EXPORTS = ["lsp_workspace_bytes", "lsp_kv_cache_bytes", "lsp_init", "lsp_set_sched", "lsp_set_option",
            "lsp_begin", "lsp_denoise_step", "lsp_commit", "lsp_generate", "lsp_generate_host", "lsp_active", "lsp_score_rows",
-           "lsp_get_scores", "lsp_head_scan", "lsp_scan", "lsp_op_linear", "lsp_last_timing", "lsp_get_counters", "lsp_reset_counters",
+           "lsp_get_scores", "lsp_head_scan", "lsp_scan", "lsp_op_linear", "lsp_op_attention", "lsp_last_timing", "lsp_get_counters", "lsp_reset_counters",
            "lsp_linear_static", "lsp_last_error", "lsp_destroy"]
 
 
@@ -73,6 +73,8 @@ def _load():
     l.lsp_head_scan.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int] + [C.c_void_p] * 4
     l.lsp_scan.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int] + [C.c_void_p] * 4
     l.lsp_op_linear.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int]
+    l.lsp_op_attention.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                   C.c_int]
     l.lsp_last_timing.argtypes = [C.c_void_p, C.c_void_p]
     l.lsp_get_counters.argtypes = [C.c_void_p, C.c_void_p]
     l.lsp_reset_counters.argtypes = [C.c_void_p]
@@ -289,17 +291,30 @@ class LSPDecoder:
                                       out.data_ptr(), M, N, K))
         return out
 
+    def op_attention(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, out: torch.Tensor,
+                     cache_len, rows):
+        """One layer's suffix-over-prefix attention on packed rows; the cached K/V are read from kv_view()."""
+        cl = np.ascontiguousarray(cache_len, dtype=np.int32)
+        rw = np.ascontiguousarray(rows, dtype=np.int32)
+        assert cl.shape == rw.shape and q.shape[0] == int(rw.sum()) == k_new.shape[0] == v_new.shape[0] == out.shape[0]
+        for t in (q, k_new, v_new, out):
+            assert t.is_cuda and t.is_contiguous() and t.dtype == self.tdtype
+        self._check(lib.lsp_op_attention(self._h, layer, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
+                                         cl.ctypes.data, rw.ctypes.data, len(cl)))
+        return out
+
     def last_timing(self):
         a = np.zeros(8, dtype=np.float32)
         self._check(lib.lsp_last_timing(self._h, a.ctypes.data))
         return a
 
     def counters(self):
-        a = np.zeros(16, dtype=np.float64)
+        a = np.zeros(18, dtype=np.float64)
         self._check(lib.lsp_get_counters(self._h, a.ctypes.data))
         return dict(zip(("launches", "gemm_bytes", "gemm_flops", "attn_bytes", "append_bytes", "head_bytes",
                          "head_flops", "steps", "launches_misc", "launches_gemm", "launches_attn", "launches_head",
-                         "launches_scan", "launches_commit", "attn_flops", "tokens"), a.tolist()))
+                         "launches_scan", "launches_commit", "attn_flops", "tokens", "attn_kernel", "attn_cluster"),
+                        a.tolist()))
 
     def reset_counters(self):
         self._check(lib.lsp_reset_counters(self._h))

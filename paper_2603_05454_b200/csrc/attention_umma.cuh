@@ -254,6 +254,18 @@ k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ 
 #pragma unroll
         for (int i = 0; i < AU_BN; ++i)
           if (i >= valid_keys) sv[i] = -INFINITY;
+        // The tile's V rows past the last key hold whatever lies behind it in the plane (cache rows the library never
+        // wrote, another sequence's staged rows), and 0 x NaN = NaN would reach every output row through P V.  Thread r
+        // clears key row r of the V stage (128 bytes in each of its two atoms; the swizzle only permutes within a row).
+        // The stage cannot be refilled before this tile's P is published below, so the completed phase is still current.
+        if (r >= valid_keys && mbar_wait(bar(s), (uint32_t)(t >> 1) & 1u, abort_flag)) {
+          uint8_t* vrow = KVs + (size_t)s * 2 * AU_TILE + AU_TILE + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            *reinterpret_cast<uint4*>(vrow + 16 * c) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(vrow + AU_ATOM + 16 * c) = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
       }
       float mx = -INFINITY;
 #pragma unroll

@@ -60,12 +60,13 @@ struct lsp_ctx {
   bool proposed = false;
   int score_rows = 0;
   int last_M = 0;
+  int last_attn_kernel = 0, last_attn_cluster = 1;   // what the last attention launch was (see lsp_get_counters)
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   float timing_ms[8] = {0};
   std::vector<cudaEvent_t> seg_ev;      // per-class timing: pairs of events, created on demand
   std::vector<int> seg_cls;
   int seg_n = 0;
-  double counters[16] = {0};            // see lsp_get_counters
+  double counters[18] = {0};            // see lsp_get_counters (16, 17 are filled on read)
   std::string err;
 #ifndef LSP_NO_UMMA
   UmmaState umma;
@@ -302,6 +303,78 @@ int check_status(lsp_ctx* c) {
   return LSP_OK;
 }
 
+// Suffix-over-prefix attention of layer l (Sec. 3.2: every query row of the pass sees the cached prefix [0, F_b) and all
+// of the pass's own rows).  Reads the uploaded descriptor (F, row_off), Q from q, K/V from the cache and the staging
+// planes of layer l; writes out.  max_q: most query rows of one sequence; max_keys: most keys of one sequence.
+template <typename T>
+int run_attention(lsp_ctx* c, int l, const T* Qb, T* Att, int B, int maxQ, int max_keys) {
+  const lsp_model_cfg& m = c->m;
+  const StepDesc sd = desc_of(c);
+  const int dh = m.head_dim, kvd = m.n_kv_heads * dh;
+  const size_t plane = (size_t)c->max_rows * kvd;
+  const size_t cplane = (size_t)c->max_batch * c->max_len * kvd;
+  const T* stK = (const T*)c->stage + (size_t)(2 * l) * plane;
+  const T* stV = stK + plane;
+  const T* cK = (const T*)c->kv_cache + (size_t)(2 * l) * cplane;
+  const T* cV = cK + cplane;
+  const float scale = 1.0f / sqrtf((float)dh);
+  count_launch(c, CLS_ATTN);
+  seg_begin(c, CLS_ATTN);
+  bool done = false;
+  c->last_attn_kernel = 0;
+  c->last_attn_cluster = 1;
+#ifndef LSP_NO_UMMA
+  if constexpr (std::is_same<T, bf16>::value) {
+    // the tcgen05 kernel (128-row tiles; with few CTAs the keys of a row tile are split over a cluster); a row-count
+    // threshold can send small passes to the 64-row mma.sync kernel instead
+    if (c->attn_impl == 2 && dh == 128 && !c->attn_maps.empty() && maxQ * (m.n_heads / m.n_kv_heads) >= c->attn_umma_min_rows) {
+      const int G = m.n_heads / m.n_kv_heads;
+      const int row_tiles = (maxQ * G + AU_BM - 1) / AU_BM;
+      // few CTAs: split every row tile's keys over a cluster of 2, 4 or 8 CTAs (merged through DSMEM)
+      int cl = 1;
+      if (c->attn_cluster) {
+        const int key_tiles = (max_keys + AU_BN - 1) / AU_BN;
+        const int ctas = row_tiles * m.n_kv_heads * B;
+        // ... as long as that many clusters can be resident at once (this kernel, too, runs one CTA per SM)
+        while (cl < 8 && 2 * cl * ctas <= c->umma.n_sm && 2 * cl <= key_tiles && ctas <= c->umma.max_clusters[2 * cl]) cl *= 2;
+      }
+      dim3 g3(row_tiles * cl, m.n_kv_heads, B);
+      const float sl2 = scale * 1.4426950408889634f;
+      const CUtensorMap* mp = &c->attn_maps[4 * l];
+      launch_k(c->pdl, k_attn_umma, g3, dim3(AU_THREADS), (size_t)AU_SMEM, c->stream, cl, mp[0], mp[1], mp[2], mp[3],
+               (const bf16*)Qb, Att, sd, m.n_heads, m.n_kv_heads, c->max_len, sl2, cl, c->d_status);
+      c->last_attn_kernel = 2;
+      c->last_attn_cluster = cl;
+      done = true;
+    }
+  }
+#endif
+  if constexpr (std::is_same<T, bf16>::value) {
+    if (!done && c->attn_impl >= 1) {
+      const int G = m.n_heads / m.n_kv_heads;
+      dim3 g2((maxQ * G + AM_BM - 1) / AM_BM, m.n_kv_heads, B);
+      const float sl2 = scale * 1.4426950408889634f;
+      if (dh == 128)
+        launch_k(c->pdl, k_attn_mma<128>, dim3(g2), dim3(128), attn_mma_smem_bytes<128>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
+      else
+        launch_k(c->pdl, k_attn_mma<64>, dim3(g2), dim3(128), attn_mma_smem_bytes<64>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
+      c->last_attn_kernel = 1;
+      done = true;
+    }
+  }
+  dim3 grid((maxQ + AS_BQ - 1) / AS_BQ, m.n_heads, B);
+  if (done) {
+  } else if (dh == 128)
+    launch_k(c->pdl, k_attn_simt<T, 128>, dim3(grid), dim3(128), 0, c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
+                                                     (size_t)c->max_len * kvd, scale);
+  else
+    launch_k(c->pdl, k_attn_simt<T, 64>, dim3(grid), dim3(128), 0, c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
+                                                    (size_t)c->max_len * kvd, scale);
+  seg_end(c);
+  CU(cudaGetLastError());
+  return LSP_OK;
+}
+
 template <typename T>
 int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   const lsp_model_cfg& m = c->m;
@@ -320,7 +393,6 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
     h[3 * s + b] = M;
     h[4 * s + b] = Mh;
     h[5 * s + b] = c->Fp[b];
-    h[6 * s + b] = 0;
     M += rows;
     Mh += c->N[b];
     if (rows > maxQ) maxQ = rows;
@@ -330,7 +402,9 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   if (M == 0) return fail(c, LSP_ERR_STATE, "lsp_denoise_step: every sequence is already fully committed");
   const auto host_t0 = std::chrono::steady_clock::now();
   CU(cudaEventRecord(c->ev0, c->stream));
-  CU(cudaMemcpyAsync(c->d_desc, h, 7 * (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
+  // the step owns the first six arrays; the seventh (commit lengths) belongs to lsp_commit, whose upload from the same
+  // pinned mirror may still be in flight
+  CU(cudaMemcpyAsync(c->d_desc, h, 6 * (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
   const StepDesc sd = desc_of(c);
   const int d = m.d_model, dh = m.head_dim, qd = m.n_heads * dh, kvd = m.n_kv_heads * dh;
   T* X = (T*)c->X;
@@ -351,13 +425,9 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   seg_end(c);
   count_launch(c, CLS_MISC);
   const size_t plane = (size_t)c->max_rows * kvd;           // elements per staged (layer, K|V) plane
-  const size_t cplane = (size_t)c->max_batch * c->max_len * kvd;
-  const float scale = 1.0f / sqrtf((float)dh);
   for (int l = 0; l < m.n_layers; ++l) {
     T* stK = (T*)c->stage + (size_t)(2 * l) * plane;
     T* stV = stK + plane;
-    const T* cK = (const T*)c->kv_cache + (size_t)(2 * l) * cplane;
-    const T* cV = cK + cplane;
     seg_begin(c, CLS_MISC);
     launch_k(c->pdl, k_rmsnorm<T>, dim3(M), dim3(256), 0, c->stream, X, (const T*)c->attn_norm[l], Nrm, nullptr, d, m.rms_eps);
     seg_end(c);
@@ -377,58 +447,11 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
         c->counters[CNT_ATTN_BYTES] += (2.0 * (c->F[b] + rows_b) * kvd + 2.0 * rows_b * qd) * sizeof(T);
         c->counters[CNT_ATTN_FLOPS] += 4.0 * rows_b * (c->F[b] + rows_b) * qd;
       }
-      count_launch(c, CLS_ATTN);
-      seg_begin(c, CLS_ATTN);
-      bool done = false;
-#ifndef LSP_NO_UMMA
-      if constexpr (std::is_same<T, bf16>::value) {
-        // the tcgen05 kernel (128-row tiles; with few CTAs the keys of a row tile are split over a cluster); a row-count
-        // threshold can send small passes to the 64-row mma.sync kernel instead
-        if (c->attn_impl == 2 && dh == 128 && !c->attn_maps.empty() && maxQ * (m.n_heads / m.n_kv_heads) >= c->attn_umma_min_rows) {
-          const int G = m.n_heads / m.n_kv_heads;
-          const int row_tiles = (maxQ * G + AU_BM - 1) / AU_BM;
-          // few CTAs: split every row tile's keys over a cluster of 2, 4 or 8 CTAs (merged through DSMEM)
-          int cl = 1;
-          if (c->attn_cluster) {
-            int max_keys = 0;
-            for (int b = 0; b < B; ++b)
-              if (c->N[b] > 0) max_keys = std::max(max_keys, c->F[b] + c->pend[b] + (scattered ? c->G[b] : c->N[b]));
-            const int key_tiles = (max_keys + AU_BN - 1) / AU_BN;
-            const int ctas = row_tiles * m.n_kv_heads * B;
-            // ... as long as that many clusters can be resident at once (this kernel, too, runs one CTA per SM)
-            while (cl < 8 && 2 * cl * ctas <= c->umma.n_sm && 2 * cl <= key_tiles && ctas <= c->umma.max_clusters[2 * cl]) cl *= 2;
-          }
-          dim3 g3(row_tiles * cl, m.n_kv_heads, B);
-          const float sl2 = scale * 1.4426950408889634f;
-          const CUtensorMap* mp = &c->attn_maps[4 * l];
-          launch_k(c->pdl, k_attn_umma, g3, dim3(AU_THREADS), (size_t)AU_SMEM, c->stream, cl, mp[0], mp[1], mp[2], mp[3],
-                   (const bf16*)Qb, Att, sd, m.n_heads, m.n_kv_heads, c->max_len, sl2, cl, c->d_status);
-          done = true;
-        }
-      }
-#endif
-      if constexpr (std::is_same<T, bf16>::value) {
-        if (!done && c->attn_impl >= 1) {
-          const int G = m.n_heads / m.n_kv_heads;
-          dim3 g2((maxQ * G + AM_BM - 1) / AM_BM, m.n_kv_heads, B);
-          const float sl2 = scale * 1.4426950408889634f;
-          if (dh == 128)
-            launch_k(c->pdl, k_attn_mma<128>, dim3(g2), dim3(128), attn_mma_smem_bytes<128>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
-          else
-            launch_k(c->pdl, k_attn_mma<64>, dim3(g2), dim3(128), attn_mma_smem_bytes<64>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
-          done = true;
-        }
-      }
-      dim3 grid((maxQ + AS_BQ - 1) / AS_BQ, m.n_heads, B);
-      if (done) {
-      } else if (dh == 128)
-        launch_k(c->pdl, k_attn_simt<T, 128>, dim3(grid), dim3(128), 0, c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
-                                                         (size_t)c->max_len * kvd, scale);
-      else
-        launch_k(c->pdl, k_attn_simt<T, 64>, dim3(grid), dim3(128), 0, c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
-                                                        (size_t)c->max_len * kvd, scale);
-      seg_end(c);
-      CU(cudaGetLastError());
+      int max_keys = 0;
+      for (int b = 0; b < B; ++b)
+        if (c->N[b] > 0) max_keys = std::max(max_keys, c->F[b] + c->pend[b] + (scattered ? c->G[b] : c->N[b]));
+      const int rc = run_attention<T>(c, l, Qb, Att, B, maxQ, max_keys);
+      if (rc) return rc;
     }
     {
       EpiResidual<T> e{X, d};
@@ -934,6 +957,42 @@ int lsp_op_linear(lsp_ctx* c, int op, const void* A, const void* W, const void* 
   return check_status(c);
 }
 
+int lsp_op_attention(lsp_ctx* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
+                     const int32_t* cache_len, const int32_t* rows, int batch) {
+  if (!c || !q || !k_new || !v_new || !out || !cache_len || !rows) return LSP_ERR_ARG;
+  if (layer < 0 || layer >= c->m.n_layers || batch < 1 || batch > c->max_batch)
+    return fail(c, LSP_ERR_ARG, "lsp_op_attention: layer %d or batch %d out of range", layer, batch);
+  const int s = c->max_batch + 1;
+  int* h = c->h_desc;
+  int M = 0, maxQ = 0, max_keys = 0;
+  for (int b = 0; b < batch; ++b) {
+    if (cache_len[b] < 0 || rows[b] < 0 || cache_len[b] + rows[b] > c->max_len)
+      return fail(c, LSP_ERR_ARG, "lsp_op_attention: sequence %d has %d cached + %d new positions, more than max_len %d", b,
+                  cache_len[b], rows[b], c->max_len);
+    h[0 * s + b] = cache_len[b];
+    h[3 * s + b] = M;
+    M += rows[b];
+    maxQ = std::max(maxQ, rows[b]);
+    if (rows[b] > 0) max_keys = std::max(max_keys, cache_len[b] + rows[b]);
+  }
+  h[3 * s + batch] = M;
+  c->proposed = false;                 // the descriptor of a pending lsp_denoise_step is overwritten
+  if (M == 0) return LSP_OK;
+  CU(cudaMemcpyAsync(c->d_desc, h, (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
+  CU(cudaMemcpyAsync(c->d_desc + 3 * s, h + 3 * s, (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
+  const size_t kvd = (size_t)c->m.n_kv_heads * c->m.head_dim;
+  const size_t plane = (size_t)c->max_rows * kvd * c->esz;
+  char* stK = c->stage + (size_t)(2 * layer) * plane;
+  CU(cudaMemcpyAsync(stK, k_new, (size_t)M * kvd * c->esz, cudaMemcpyDeviceToDevice, c->stream));
+  CU(cudaMemcpyAsync(stK + plane, v_new, (size_t)M * kvd * c->esz, cudaMemcpyDeviceToDevice, c->stream));
+  const int rc = c->m.dtype == 0 ? run_attention<float>(c, layer, (const float*)q, (float*)out, batch, maxQ, max_keys)
+                                 : run_attention<bf16>(c, layer, (const bf16*)q, (bf16*)out, batch, maxQ, max_keys);
+  if (rc) return rc;
+  CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaStreamSynchronize(c->stream));
+  return check_status(c);
+}
+
 int lsp_last_timing(lsp_ctx* c, float* ms) {
   if (!c || !ms) return LSP_ERR_ARG;
   CU(cudaStreamSynchronize(c->stream));
@@ -944,6 +1003,8 @@ int lsp_last_timing(lsp_ctx* c, float* ms) {
 
 int lsp_get_counters(lsp_ctx* c, double* out) {
   if (!c || !out) return LSP_ERR_ARG;
+  c->counters[16] = c->last_attn_kernel;
+  c->counters[17] = c->last_attn_cluster;
   memcpy(out, c->counters, sizeof c->counters);
   return LSP_OK;
 }

@@ -1,0 +1,105 @@
+"""K4 parity at the kernel level: the suffix-over-prefix attention (Sec. 3.2) through lsp_op_attention against
+oracle.dlm.attention, element by element, at head shapes of the benchmark models and at the launch shapes the decodes
+take: key tiles split over thread block clusters of 2, 4 and 8 CTAs, grouped-query packing that crosses a 128-row tile,
+cache lengths that are not a multiple of the key tile, staged blocks that straddle a key tile, ragged batches."""
+import numpy as np
+import pytest
+import torch
+
+import lsp_synth as S
+from oracle import dlm
+from gpu_util import DEV
+
+pytestmark = pytest.mark.gpu
+
+# The kernel feeds bf16 softmax weights (relative error 2^-9 each) to the tensor core and rounds the output once; the
+# oracle keeps the weights in fp64.  With |v| <= 4.9 (the generator's support) and independent errors over the keys the
+# difference stays far below 2^-8 * max|v| = 1.9e-2: the bound asserted is the benchmark's 2e-2 absolute, and the
+# measured maximum is printed (pytest -s) and asserted against a tighter, measured ceiling.
+ATOL = 2e-2
+MEASURED_CEILING = 8e-3
+
+
+def _run_case(hq, hkv, cache_len, rows, max_len, attn_impl=None, expect_cluster=None, seed=0, poison=False):
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+    dh, B = 128, len(rows)
+    sh = S.ModelShape(1, 128 * hq, hq, hkv, dh, 64, 256, dtype="bf16")
+    z = lambda *s: torch.zeros(*s, dtype=torch.bfloat16, device=DEV)
+    d = sh.d_model
+    w = dict(embed=z(256, d), w_head=z(256, d), final_norm=z(d),
+             layers=[dict(attn_norm=z(d), w_qkv=z((hq + 2 * hkv) * dh, d), w_o=z(d, hq * dh), ffn_norm=z(d), w_gate=z(64, d),
+                          w_up=z(64, d), w_down=z(d, 64))])
+    dec = LSPDecoder(sh, w, SchedCfg(), B, max_len, device=DEV)
+    if attn_impl is not None:
+        dec.set_option(1, attn_impl)
+    M = int(sum(rows))
+    bf = torch.bfloat16
+    q = S.normal((M, hq * dh), seed, 1, 1.0, bf, DEV)
+    kn = S.normal((M, hkv * dh), seed, 2, 1.0, bf, DEV)
+    vn = S.normal((M, hkv * dh), seed, 3, 1.0, bf, DEV)
+    kv = dec.kv_view()                                   # [1, 2, B, max_len, hkv, dh]
+    if poison:
+        # NaN bit patterns wherever the library has not written: cache rows past each prefix and the whole staging area
+        kv.view(torch.int16).fill_(0x7FC0)
+        stage_bytes = 2 * B * max_len * hkv * dh * 2
+        dec.workspace[-((stage_bytes + 255) // 256 * 256):].view(torch.int16).fill_(0x7FC0)
+    ck = S.normal((B, max_len, hkv, dh), seed, 4, 1.0, bf, DEV)
+    cv = S.normal((B, max_len, hkv, dh), seed, 5, 1.0, bf, DEV)
+    for b in range(B):
+        kv[0, 0, b, :cache_len[b]] = ck[b, :cache_len[b]]
+        kv[0, 1, b, :cache_len[b]] = cv[b, :cache_len[b]]
+    out = torch.full((M, hq * dh), float("nan"), dtype=bf, device=DEV)
+    dec.op_attention(0, q, kn, vn, out, cache_len, rows)
+    cnt = dec.counters()
+    dec.close()
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    got = f64(out)
+    qn, knn, vnn, ckn, cvn = f64(q), f64(kn), f64(vn), f64(ck), f64(cv)
+    worst, r0 = 0.0, 0
+    for b in range(B):
+        Q, F = rows[b], cache_len[b]
+        if Q == 0:
+            continue
+        k_all = np.concatenate([ckn[b, :F], knn[r0:r0 + Q].reshape(Q, hkv, dh)], axis=0)
+        v_all = np.concatenate([cvn[b, :F], vnn[r0:r0 + Q].reshape(Q, hkv, dh)], axis=0)
+        ref = dlm.round_bf16(dlm.attention(qn[r0:r0 + Q].reshape(Q, hq, dh), k_all, v_all)).reshape(Q, hq * dh)
+        g = got[r0:r0 + Q]
+        assert np.isfinite(g).all(), f"sequence {b}: non-finite output"
+        worst = max(worst, float(np.abs(g - ref).max()))
+        r0 += Q
+    print(f"attention hq={hq} hkv={hkv} F={cache_len} rows={rows}: kernel {int(cnt['attn_kernel'])}, cluster "
+          f"{int(cnt['attn_cluster'])}, max |err| {worst:.2e}")
+    assert worst <= ATOL, worst
+    assert worst <= MEASURED_CEILING, worst
+    if expect_cluster is not None:
+        assert int(cnt["attn_kernel"]) == 2 and int(cnt["attn_cluster"]) == expect_cluster, cnt
+    return worst, cnt
+
+
+@pytest.mark.parametrize("case", [
+    # (hq, hkv, cache lengths, rows, max_len, expected cluster size)
+    (32, 32, [412], [100], 512, 4),          # the LLaDA-shaped steady state: 32 CTAs, 4 key tiles -> clusters of 4
+    (28, 4, [2032], [16], 2048, 8),          # the Dream shape late in a decode: 4 CTAs, 16 key tiles -> clusters of 8
+    (28, 4, [300], [40], 384, 2),            # grouped 7:1, 280 (query, head) rows: three row tiles, the group straddles tiles
+    (32, 32, [77], [200], 320, 2),           # staged block over two key tiles, the cache tile ragged; 64 CTAs -> pairs
+    (8, 2, [0], [130], 256, None),           # no cache at all (the first pass), a ragged second staged tile
+    (8, 2, [129, 5, 250], [3, 0, 60], 320, None),      # ragged batch, one finished sequence (no rows)
+    (4, 4, [640], [1], 768, None),           # a single query row over six key tiles
+])
+def test_attention_tcgen05_against_the_oracle(case):
+    hq, hkv, F, rows, max_len, cl = case
+    _run_case(hq, hkv, F, rows, max_len, expect_cluster=cl)
+
+
+@pytest.mark.parametrize("attn_impl", [0, 1])
+def test_attention_other_kernels_against_the_oracle(attn_impl):
+    """The CUDA-core and mma.sync kernels on the same cases (they serve fp32 models and head_dim 64)."""
+    _run_case(8, 2, [129, 5], [33, 70], 256, attn_impl=attn_impl)
+
+
+def test_attention_ignores_memory_it_never_wrote():
+    """Cache rows past the prefix and staging rows past the pass hold NaN bit patterns (memory the caller handed over
+    uninitialised): a ragged last key tile brings such rows into shared memory, and they must not reach the output."""
+    _run_case(32, 32, [412], [100], 700, seed=3, poison=True)
+    _run_case(28, 4, [300, 17], [40, 9], 500, seed=4, poison=True)
+    _run_case(8, 2, [129, 5, 250], [3, 0, 60], 320, attn_impl=1, seed=5, poison=True)

@@ -117,3 +117,49 @@ def test_bf16_mode_rounds_at_declared_points():
     _, k_new, v_new = m.forward(np.array([1, 2, 49]), np.arange(3), ck, cv, [2])
     for a in k_new + v_new:
         assert np.array_equal(a, dlm.round_bf16(a))
+
+
+def test_bf16_mode_rounding_points_are_exactly_the_declared_ones(monkeypatch):
+    """One forward pass of a bf16 model, with every call of the rounding hook recorded and the inputs of the norm and
+    attention routines captured.  Declared points, per layer: norm output, Q, K, V (after the rotation), attention
+    output, residual update, second norm output, SwiGLU product, second residual update; then the final norm.  Logits
+    and softmax weights stay unrounded.  A dropped (or added) rounding changes the recorded sequence."""
+    sh = _tiny(dtype="bf16")
+    sh.n_layers = 2
+    m = dlm.OracleDLM(sh, S.make_weights(sh, 2))
+    Q, head_rows = 5, [2, 4]
+    is_bf16 = lambda a: np.array_equal(a, dlm.round_bf16(a))
+    calls = []
+    orig_r = m.r
+    m.r = lambda x: calls.append((np.shape(x), is_bf16(x))) or orig_r(x)
+    seen = {"norm_in": [], "attn_in": []}
+    o_norm, o_attn = dlm.rms_norm, dlm.attention
+    monkeypatch.setattr(dlm, "rms_norm", lambda x, g, e: seen["norm_in"].append(is_bf16(x)) or o_norm(x, g, e))
+    monkeypatch.setattr(dlm, "attention",
+                        lambda q, k, v: seen["attn_in"].append(is_bf16(q) and is_bf16(k) and is_bf16(v)) or o_attn(q, k, v))
+    ck, cv = m.empty_cache()
+    logits, k_new, v_new = m.forward(np.array([1, 2, 49, 7, 49]), np.arange(Q), ck, cv, head_rows)
+    d, f = sh.d_model, sh.d_ffn
+    hq, hkv, dh = sh.n_heads, sh.n_kv_heads, sh.head_dim
+    per_layer = [(Q, d), (Q, hq, dh), (Q, hkv, dh), (Q, hkv, dh), (Q, hq, dh), (Q, d), (Q, d), (Q, f), (Q, d)]
+    assert [c[0] for c in calls] == per_layer * sh.n_layers + [(len(head_rows), d)]
+    assert not any(c[1] for c in calls)                   # every rounding did something: its input was not bf16 yet
+    assert all(seen["norm_in"]) and len(seen["norm_in"]) == 2 * sh.n_layers + 1     # residual stream is bf16 at every norm
+    assert all(seen["attn_in"]) and len(seen["attn_in"]) == sh.n_layers             # Q, K, V are bf16 when attention reads them
+    assert not is_bf16(logits)                            # logits are accumulators, never rounded
+    for a in k_new + v_new:
+        assert is_bf16(a)
+    # softmax weights are not rounded: attention() never reaches the rounding routine
+    def boom(x):
+        raise AssertionError("attention rounded something")
+    monkeypatch.setattr(dlm, "round_bf16", boom)
+    rng = np.random.default_rng(0)
+    o_attn(rng.normal(size=(3, hq, dh)), rng.normal(size=(4, hkv, dh)), rng.normal(size=(4, hkv, dh)))
+
+
+def test_fp32_mode_rounds_nothing():
+    sh = _tiny(dtype="fp32")
+    m = dlm.OracleDLM(sh, S.make_weights(sh, 2))
+    ck, cv = m.empty_cache()
+    x = np.random.default_rng(1).normal(size=(3, 7))
+    assert m.r(x) is x

@@ -24,15 +24,22 @@ def definitional(passes, delims, l_min, W):
     return Lp, min(N, max(1, L))
 
 
-@pytest.mark.parametrize("N", [1, 2, 3, 5, 8, 10])
+def _delimiter_patterns(N):
+    """Every delimiter pattern up to N = 8; beyond that five fixed patterns plus eight seeded random ones."""
+    if N <= 8:
+        return list(itertools.product((0, 1), repeat=N))
+    rng = np.random.default_rng(1000 + N)
+    fixed = [tuple(int((i * 7 + k) % 3 == 0) for i in range(N)) for k in range(3)] + [(0,) * N, (1,) * N]
+    return fixed + [tuple(int(x) for x in rng.integers(0, 2, N)) for _ in range(8)]
+
+
+@pytest.mark.parametrize("N", list(range(1, 13)))
 def test_scan_brute_force_all_patterns(N):
     for W in (0, 1, 2, 16, -1):
         for l_min in (1, 3):
             for passes in itertools.product((0, 1), repeat=N):
                 score = [0.95 if p else 0.10 for p in passes]
-                for delims in itertools.product((0, 1), repeat=N) if N <= 5 else \
-                        [tuple((i * 7 + k) % 3 == 0 for i in range(N)) for k in range(3)] + \
-                        [tuple(0 for _ in range(N)), tuple(1 for _ in range(N))]:
+                for delims in _delimiter_patterns(N):
                     yhat = [1 if d else 100 for d in delims]
                     r = S.lsp_scan(score, yhat, lambda t: t == 1, tau=0.9, l_min=l_min, W=W)
                     Lp, L = definitional(passes, delims, l_min, W)

@@ -84,3 +84,19 @@ def test_flip_counts_helper_matches_decode_records():
     fc = flip_counts([(r["masked"], r["yhat"]) for r in recs])
     assert fc == [(r["flips"], r["flip_base"]) for r in recs]
     assert flip_counts([([1, 2, 3], [5, 6, 7]), ([2, 3], [6, 9]), ([3], [9])]) == [(0, 0), (1, 2), (0, 1)]
+
+
+def test_flip_counts_hand_examples():
+    """Worked by hand.  A position counts in the base only if it was masked (scored) at the step before as well; it
+    flips when its argmax differs between the two."""
+    # step 0: nothing scored before.  step 1: positions 10..13 were all scored at step 0 -> base 4; 11 and 13 changed.
+    # step 2: 12, 13 carried over, both changed; 20 is new (not in the base).
+    assert flip_counts([([10, 11, 12, 13], [1, 2, 3, 4]),
+                        ([10, 11, 12, 13], [1, 9, 3, 8]),
+                        ([12, 13, 20], [4, 3, 3])]) == [(0, 0), (2, 4), (2, 2)]
+    # a position that leaves the masked set and comes back is compared with the step just before only, where it was
+    # absent: it is not in the base; an unchanged survivor is in the base and does not flip
+    assert flip_counts([([0, 1], [7, 7]), ([1], [7]), ([0, 1], [5, 6])]) == [(0, 0), (0, 1), (1, 1)]
+    # prefix decode that commits one position per step with stable predictions: base N-1, N-2, ... and no flips
+    steps = [(list(range(k, 6)), [40 + p for p in range(k, 6)]) for k in range(6)]
+    assert flip_counts(steps) == [(0, 0)] + [(0, 6 - k) for k in range(1, 6)]
