@@ -272,7 +272,7 @@ def run_gemm_chain(dec, w, sh, M, dev, reps=3):
     x = torch.zeros(M, d, dtype=bf, device=dev)
     o_qkv = torch.empty(M, qd + 2 * kvd, dtype=bf, device=dev)
     h_f = torch.empty(M, f, dtype=bf, device=dev)
-    dec.set_option(3, 1)                                   # queue only; no synchronisation per call
+    dec.debug_set(3, 1)                                   # queue only; no synchronisation per call
 
     def chain():
         for lw in dec.layer_weights:
@@ -290,7 +290,7 @@ def run_gemm_chain(dec, w, sh, M, dev, reps=3):
         chain()
     ev1.record()
     torch.cuda.synchronize(dev)
-    dec.set_option(3, 0)
+    dec.debug_set(3, 0)
     dec.op_linear(0, a_d[:1], dec.layer_weights[0]["w_qkv"], None, o_qkv[:1])      # synchronising call: surfaces a device-side status
     ms = ev0.elapsed_time(ev1) / reps
     wbytes = sh.n_layers * 2.0 * ((qd + 2 * kvd) * d + d * qd + 2 * f * d + d * f)
@@ -485,7 +485,7 @@ def run_head_bench(dev, peaks, steps, warmup):
                 h2d=host_h.numel() * 2, d2h=B * L * 12, classes=class_report(cnt2, tms, peaks))
 
 
-def run_topology_compare(wl, dev, peaks, warmup):
+def run_topology_compare(wl, dev, peaks, warmup, class_passes=24):
     """cfg5: the LSP decode next to the scattered-acceptance baseline (top-k anywhere, k = 32 per step) on the same
     kernels: denoiser calls, token flips, step latency and KV-append bytes per committed token.  One timed decode per
     topology; the warm-up decodes use a 64-token generation (they warm the same kernels; a full LSP decode of this
@@ -538,8 +538,70 @@ def run_topology_compare(wl, dev, peaks, warmup):
                      "kv_append_bytes_per_committed_token": cnt["append_bytes"] / (B * G),
                      "gpu_launches": int(cnt["launches"]),
                      "rows_first_last": [sum(r["rows"] for r in recs[:B]), sum(r["rows"] for r in recs[-B:])]}
+    # per-class kernel times (one CUDA-event pair per launch) over the first passes of one more LSP decode
+    dec.set_sched(scheds["lsp"])
+    tokens[:, :P] = prompt.to(dev)
+    dec.begin(tokens, [P] * B, [G] * B)
+    dec.set_option(2, 1)
+    dec.reset_counters()
+    n_cls = 0
+    while n_cls < class_passes and dec.active()[1] > 0:
+        dec.denoise_step()
+        dec.commit()
+        n_cls += 1
+    tms = dec.last_timing()
+    cnt = dec.counters()
+    dec.set_option(2, 0)
+    classes = class_report(cnt, tms, peaks)
     dec.close()
-    return out, k
+    del dec, w
+    torch.cuda.empty_cache()
+    return out, k, classes, n_cls
+
+
+def head_line(dev, peaks, peak_kind, steps, warmup, sampler=None):
+    """cfg2 as a bench line (also used as an entry under 'also')."""
+    if sampler:
+        sampler.start()
+    r = run_head_bench(dev, peaks, steps, warmup)
+    clocks = sampler.stop() if sampler else None
+    head = r["classes"]["head"]
+    return {"metric": "scored_positions_per_s", "value": r["positions"] / (r["ms"] * 1e-3), "unit": "positions/s",
+            "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": r["ms"] / steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "cfg2: fused LM head + confidence + LSP scan, hidden [8,1024,4096], vocab 126464",
+                       "l2": "inputs_exceed_l2 (1.04 GB head weight)"},
+            "roofline": {"bound": "tensor", "achieved": head.get("tflops"), "peak": peaks["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": (head.get("tflops") or 0) / peaks["bf16_tflops"],
+                         "traffic": head.get("traffic"), "peak_kind": "burst, of " + peak_kind,
+                         "kernel": "k_gemm_stream<256,.,.,EpiHead> (LM head with the top-2 / log-sum-exp reduction in its epilogue)"},
+            "e2e": {"value": r["positions"] / (r["e2e_ms"] * 1e-3), "unit": "positions/s",
+                    "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"]},
+            "gpu_launches": r["launches"], "classes": r["classes"], "clocks": clocks}
+
+
+def topology_line(wl, dev, peaks, peak_kind, warmup, sampler=None):
+    """cfg5 as a bench line (also used as an entry under 'also'): one timed decode per topology."""
+    if sampler:
+        sampler.start()
+    cmp_, k, classes, n_cls = run_topology_compare(wl, dev, peaks, warmup)
+    clocks = sampler.stop() if sampler else None
+    lsp = cmp_["lsp"]
+    g = classes["gemm"]
+    tc = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    return {"metric": "committed_tokens_per_s", "value": lsp["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1, "steps": 1,
+            "warmup": warmup, "ms_per_step": lsp["decode_ms"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"cfg5: LLaDA-8B shape, batch {wl.batch}, prompt {wl.prompt_len} + {wl.gen_len} masked, "
+                                   f"LSP (tau {wl.tau}) next to scattered top-{k} acceptance, random init",
+                       "warmup_decodes": "64-token generations", "head_scale": wl.shape.head_scale,
+                       "l2": "inputs_exceed_l2"},
+            "roofline": {"bound": "tensor", "achieved": g.get("tflops"), "peak": tc, "unit": "TFLOP/s",
+                         "frac": g.get("tensor_frac_sustained"), "traffic": g.get("traffic"),
+                         "peak_kind": "sustained, of " + peak_kind,
+                         "kernel": "k_gemm_stream (layer GEMMs; 17 k to 33 k rows per pass: tensor-bound)",
+                         "timed": f"per-launch CUDA events over the first {n_cls} passes of one more LSP decode"},
+            "classes": classes, "topologies": cmp_, "gpu_launches": lsp["gpu_launches"], "clocks": clocks}
 
 
 def main():
@@ -549,7 +611,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="own", choices=["own", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
-    ap.add_argument("--also", default="cfg4", help="second workload reported under 'also' at N=1 ('none' to skip)")
+    ap.add_argument("--also", default="cfg4,cfg2,cfg5",
+                    help="further workloads reported under 'also' at N=1, comma-separated ('none' to skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -579,39 +642,12 @@ def main():
     sampler = ClockSampler(uuid)
 
     if args.workload == "cfg2":
-        sampler.start()
-        r = run_head_bench(dev, peaks, args.steps, args.warmup)
-        clocks = sampler.stop()
-        head = r["classes"]["head"]
-        line = {"metric": "scored_positions_per_s", "value": r["positions"] / (r["ms"] * 1e-3), "unit": "positions/s",
-                "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["ms"] / args.steps,
-                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": "cfg2: fused LM head + confidence + LSP scan, hidden [8,1024,4096], vocab 126464",
-                           "l2": "inputs_exceed_l2 (1.04 GB head weight)"},
-                "roofline": {"bound": "tensor", "achieved": head.get("tflops"), "peak": peaks["bf16_tflops"],
-                             "unit": "TFLOP/s", "frac": (head.get("tflops") or 0) / peaks["bf16_tflops"],
-                             "traffic": head.get("traffic"), "peak_kind": "burst, of " + peak_kind},
-                "e2e": {"value": r["positions"] / (r["e2e_ms"] * 1e-3), "unit": "positions/s",
-                        "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"]},
-                "gpu_launches": r["launches"], "classes": r["classes"], "clocks": clocks}
-        print(json.dumps(line))
+        print(json.dumps(head_line(dev, peaks, peak_kind, args.steps, args.warmup, sampler)))
         return 0
 
     wl = S.config(args.workload)
     if args.workload == "cfg5":
-        sampler.start()
-        cmp_, k = run_topology_compare(wl, dev, peaks, args.warmup)
-        clocks = sampler.stop()
-        lsp = cmp_["lsp"]
-        line = {"metric": "committed_tokens_per_s", "value": lsp["tokens_per_s"], "unit": "tokens/s", "n_gpus": 1, "steps": 1,
-                "warmup": args.warmup, "ms_per_step": lsp["decode_ms"], "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": f"cfg5: LLaDA-8B shape, batch {wl.batch}, prompt {wl.prompt_len} + {wl.gen_len} masked, "
-                                       f"LSP (tau {wl.tau}) next to scattered top-{k} acceptance, random init",
-                           "warmup_decodes": "64-token generations", "head_scale": wl.shape.head_scale,
-                           "l2": "inputs_exceed_l2"},
-                "topologies": cmp_, "gpu_launches": lsp["gpu_launches"], "clocks": clocks}
-        print(json.dumps(line))
+        print(json.dumps(topology_line(wl, dev, peaks, peak_kind, args.warmup, sampler)))
         return 0
     r = run_decode_bench(wl, dev, rank, world, peaks, args.steps, args.warmup, sampler, adaptive=(world == 1))
     (ms_max, e2e_max), tokens_total = reduce_replicas([r["ms"], r.get("e2e_ms", 0.0)], r["tokens"], world, dev)
@@ -652,12 +688,20 @@ def main():
             "rows": gc["rows"], "launches": gc["launches"], "ms": round(gc["ms"], 4), "achieved": round(gc["gbs"], 1),
             "unit": "GB/s", "frac": round(gc["gbs"] / peaks["hbm_gbs"], 4), "tflops": round(gc["tflops"], 1)}
 
-    if rank == 0 and world == 1 and args.also != "none" and args.also != args.workload:
-        wl2 = S.config(args.also)
+    also = [a for a in args.also.split(",") if a and a != "none" and a != args.workload] if (rank == 0 and world == 1) else []
+    line["also"] = []
+    for name in also:
+        if name == "cfg2":
+            line["also"].append(head_line(dev, peaks, peak_kind, args.steps, args.warmup))
+            continue
+        if name == "cfg5":
+            line["also"].append(topology_line(S.config("cfg5"), dev, peaks, peak_kind, args.warmup))
+            continue
+        wl2 = S.config(name)
         k2 = max(1, min(2, args.steps))
         r2 = run_decode_bench(wl2, dev, 0, 1, peaks, k2, 3, None, with_e2e=False)
         g2 = r2["classes"]["gemm"]
-        line["also"] = [{"workload": wl2.name, "batch": wl2.batch, "prompt_len": wl2.prompt_len, "gen_len": wl2.gen_len,
+        line["also"].append({"workload": wl2.name, "batch": wl2.batch, "prompt_len": wl2.prompt_len, "gen_len": wl2.gen_len,
                          "head_scale": wl2.shape.head_scale, "tau": wl2.tau, "steps": k2,
                          "value": r2["tokens"] / (r2["ms"] * 1e-3), "unit": "tokens/s",
                          "denoiser_passes_per_decode": r2["passes"] / k2,
@@ -672,7 +716,9 @@ def main():
                                                         "frac": round(r2["gemm_chain"]["tflops"] /
                                                                       peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]), 4)}
                                                        if r2.get("gemm_chain") else None)},
-                         "classes": r2["classes"]}]
+                         "classes": r2["classes"]})
+    if not line["also"]:
+        del line["also"]
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sh, om, prompt = oracle_sample_setup(wl, dev)

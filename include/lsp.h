@@ -127,34 +127,10 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
 /* Replaces the scheduler policy (allowed between steps). */
 int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
 
-/* Options: key 0 = GEMM implementation for bf16 (0 = CUDA-core reference kernels, 1 = tcgen05,
- * default 1); key 1 = attention implementation for bf16 (0 = CUDA-core, 1 = mma.sync tensor cores,
- * 2 = default: tcgen05 tensor cores for head_dim 128 when a (sequence, KV head) has at least [key 28, default 0] query rows x
- * group heads, else as 1);
- * key 2 = per-class CUDA-event timing (0 off, 1 on; see lsp_last_timing);
- * key 3 = lsp_op_linear returns without synchronising or checking the device status (1) or not (0);
- * key 4 = lsp_op_linear enqueues the operation this many times (timing aid); key 5 = repetition r reads its weights
- * at W + (r mod value) * N * K elements, so a buffer of several weight copies keeps the L2 cold;
- * tuning keys for the tcgen05 GEMM: 10 = CTAs a small-M GEMM is split into (0 = one per SM), 11 = maximum
- * pipeline stages, 12 = allow split-K (1) or not (0), 13 = CTAs per SM a weight-streaming GEMM (M <= 128) aims for,
- * 14 = fewest pipeline stages it accepts for that, 15 = its tile width for plain epilogues (32, 64 or 128),
- * 16 = GEMMs with at most 128 rows use the persistent weight-streaming kernel (1, default) or the tiled one (0),
- * 17 = grid of that kernel (0 by row count, 1 one CTA per SM with even shares, 2 a multiple of the tile count),
- * 18 = row count up to which mode 0 takes even shares, 19 = that kernel also takes 129..256 rows (1, default) or not (0),
- * 20 = its tile width for those (0 = automatic, 64, 128 or 256), 21 = 64-element K atoms per pipeline stage (0 = automatic, 1, 2),
- * 22 = fewest two-atom stages the automatic choice accepts, 23 = its tile width for up to 128 rows (0 = automatic,
- * 64, 128 or 256), 24 = row tiles per CTA it uses for more than 256 rows (1, 2,
- * 3 = automatic, default; 0 = the tiled kernel takes those), 25 = launch the step's kernels with programmatic dependent
- * launch (1, default): each kernel's set-up, and a GEMM's first weight tiles, overlap the tail of its predecessor; 0 = plain
- * launches, 26 = MMA-issuing warps of the persistent kernel with one
- * row tile per CTA (1, default, or 2), 27 = the persistent kernel caps its shared memory at half an
- * SM when three pipeline stages still fit, so that its successor can become resident beside it (1, default),
- * 28 = see key 1, 30 = the tcgen05 attention splits a row tile's keys over a thread block cluster when there are few CTAs
- * (1, default), 29 = the K slices of a split tile run as one thread block cluster and are reduced through distributed
- * shared memory (1, default) or through global scratch by the last CTA to arrive (0), 32 = tile width of the dual
- * (SwiGLU) GEMM in the persistent kernel: 0 = automatic (default), 192 or 256, 33 = a cluster of 2 exchanges half tiles
- * (1, default: each CTA keeps the half it finishes in tensor memory) or publishes whole partial tiles like larger
- * clusters (0). */
+/* Implementation switches: key 0 = GEMM implementation for bf16 models (0 = CUDA-core reference kernels, 1 = tcgen05,
+ * default 1); key 1 = attention implementation for bf16 models (0 = CUDA-core, 1 = mma.sync tensor cores, 2 = default:
+ * tcgen05 tensor cores for head_dim 128, else as 1); key 2 = per-class CUDA-event timing (0 off, 1 on; see
+ * lsp_last_timing).  Any other key: LSP_ERR_ARG. */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

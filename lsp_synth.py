@@ -159,15 +159,22 @@ def make_weights(shape: ModelShape, seed: int, device="cpu") -> Dict[str, object
         "final_norm": torch.ones(d, dtype=dt, device=device),
         "layers": [],
     }
+    for l in range(shape.n_layers):
+        w["layers"].append(make_layer(shape, seed, l, device))
+    return w
+
+
+def make_layer(shape: ModelShape, seed: int, l: int, device="cpu") -> Dict[str, torch.Tensor]:
+    """The weights of layer l alone (the same values make_weights gives), for consumers that hold one layer at a time."""
+    dt = torch.float32 if shape.dtype == "fp32" else torch.bfloat16
+    d, hq, hkv, dh, f = shape.d_model, shape.n_heads, shape.n_kv_heads, shape.head_dim, shape.d_ffn
     dims: Dict[str, Tuple[int, int]] = {
         "w_q": (hq * dh, d), "w_k": (hkv * dh, d), "w_v": (hkv * dh, d), "w_o": (d, hq * dh),
         "w_gate": (f, d), "w_up": (f, d), "w_down": (d, f)}
-    for l in range(shape.n_layers):
-        lw = {n: normal(s, seed, layer_tid(l, n), shape.w_std, dt, device) for n, s in dims.items()}
-        lw["attn_norm"] = torch.ones(d, dtype=dt, device=device)
-        lw["ffn_norm"] = torch.ones(d, dtype=dt, device=device)
-        w["layers"].append(lw)
-    return w
+    lw = {n: normal(s, seed, layer_tid(l, n), shape.w_std, dt, device) for n, s in dims.items()}
+    lw["attn_norm"] = torch.ones(d, dtype=dt, device=device)
+    lw["ffn_norm"] = torch.ones(d, dtype=dt, device=device)
+    return lw
 
 
 def make_prompt(batch: int, prompt_len: int, shape: ModelShape, seed: int, device="cpu") -> torch.Tensor:

@@ -65,18 +65,36 @@ def silu(x):
     return x / (1.0 + np.exp(-x))
 
 
+def _f64(t):
+    return np.asarray(t.float().cpu().numpy() if hasattr(t, "cpu") else t, dtype=np.float64)
+
+
 class OracleDLM:
     """Holds float64 copies of the (already dtype-rounded) weights.  Linear weights are
     [out_features, in_features]."""
 
-    def __init__(self, shape, weights):
+    def __init__(self, shape, weights, one_layer_at_a_time=False):
+        """one_layer_at_a_time: weights["layers"][l] is converted to float64 when layer l runs and dropped afterwards
+        (an 8B-parameter model is 64 GB in float64), and only the embedding rows a pass reads are converted.  Same
+        arithmetic either way."""
         self.s = shape
         self.bf16 = (shape.dtype == "bf16")
-        f64 = lambda t: np.asarray(t.float().cpu().numpy() if hasattr(t, "cpu") else t, dtype=np.float64)
-        self.embed = f64(weights["embed"])
-        self.w_head = f64(weights["w_head"])
-        self.final_norm = f64(weights["final_norm"])
-        self.layers = [{k: f64(v) for k, v in lw.items()} for lw in weights["layers"]]
+        self.w_head = _f64(weights["w_head"])
+        self.final_norm = _f64(weights["final_norm"])
+        if one_layer_at_a_time:
+            self.embed, self.layers, self._src = None, None, weights
+        else:
+            self.embed = _f64(weights["embed"])
+            self.layers = [{k: _f64(v) for k, v in lw.items()} for lw in weights["layers"]]
+
+    def layer(self, l):
+        if self.layers is not None:
+            return self.layers[l]
+        return {k: _f64(v) for k, v in self._src["layers"][l].items()}
+
+    def embed_rows(self, ids):
+        ids = np.asarray(ids, dtype=np.int64)
+        return self.embed[ids] if self.embed is not None else _f64(self._src["embed"][ids])
 
     def r(self, x):
         return round_bf16(x) if self.bf16 else x
@@ -92,9 +110,10 @@ class OracleDLM:
         Returns (logits [len(head_rows), V], k_new per layer [Q, Hkv, dh], v_new per layer)."""
         s = self.s
         Q = len(ids)
-        x = self.embed[np.asarray(ids, dtype=np.int64)]                  # [Q, d]
+        x = self.embed_rows(ids)                                         # [Q, d]
         k_new, v_new = [], []
-        for l, w in enumerate(self.layers):
+        for l in range(s.n_layers):
+            w = self.layer(l)
             n = self.r(rms_norm(x, w["attn_norm"], s.rms_eps))
             q = (n @ w["w_q"].T).reshape(Q, s.n_heads, s.head_dim)
             k = (n @ w["w_k"].T).reshape(Q, s.n_kv_heads, s.head_dim)

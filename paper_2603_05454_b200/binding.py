@@ -61,6 +61,7 @@ def _load():
                            C.c_void_p, C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_void_p]
     l.lsp_set_sched.argtypes = [C.c_void_p, C.POINTER(SchedCfgC)]
     l.lsp_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int]
+    l.lsp_debug_set.argtypes = [C.c_void_p, C.c_int, C.c_int]      # internal (csrc/lsp_tuning.h), not in EXPORTS
     l.lsp_begin.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int]
     l.lsp_denoise_step.argtypes = [C.c_void_p, C.POINTER(StepRec)]
     l.lsp_commit.argtypes = [C.c_void_p, C.c_void_p]
@@ -193,6 +194,10 @@ class LSPDecoder:
 
     def set_option(self, key: int, value: int):
         self._check(lib.lsp_set_option(self._h, key, value))
+
+    def debug_set(self, key: int, value: int):
+        """Internal tuning and benchmark knobs (csrc/lsp_tuning.h); not part of the public interface."""
+        self._check(lib.lsp_debug_set(self._h, key, value))
 
     # -- Algorithm 1
     def begin(self, tokens: torch.Tensor, prompt_len, gen_len):

@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "../../include/lsp.h"
+#include "lsp_tuning.h"
 #include "attention_mma.cuh"
 #include "attention_simt.cuh"
 #include "gemm_simt.cuh"
@@ -707,9 +708,15 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   if (!c) return LSP_ERR_ARG;
   if (key == 0) c->gemm_impl = value;
   else if (key == 1) c->attn_impl = value;
-  else if (key == 28) c->attn_umma_min_rows = value;
-  else if (key == 30) c->attn_cluster = value ? 1 : 0;
   else if (key == 2) c->timing = value;
+  else return fail(c, LSP_ERR_ARG, "lsp_set_option: unknown key %d", key);
+  return LSP_OK;
+}
+
+int lsp_debug_set(lsp_ctx* c, int key, int value) {
+  if (!c) return LSP_ERR_ARG;
+  if (key == 28) c->attn_umma_min_rows = value;
+  else if (key == 30) c->attn_cluster = value ? 1 : 0;
   else if (key == 3) c->async_ops = value;
   else if (key == 4) c->op_repeat = value < 1 ? 1 : value;
   else if (key == 5) c->op_rotate = value < 1 ? 1 : value;
@@ -736,7 +743,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   else if (key == 14) c->umma.skinny_min_stages = value < 1 ? 1 : value;
   else if (key == 15) c->umma.skinny_bn = (value == 64 || value == 32) ? value : 128;
 #endif
-  else return fail(c, LSP_ERR_ARG, "lsp_set_option: unknown key %d", key);
+  else return fail(c, LSP_ERR_ARG, "lsp_debug_set: unknown key %d", key);
   return LSP_OK;
 }
 

@@ -30,7 +30,7 @@ def _tiny_decoder(max_batch=1, max_len=8):
 def bench_gemm(M, N, K, op=0, reps=50, copies=0, warm=5, opts=()):
     dec = _tiny_decoder()
     for k, v in opts:
-        dec.set_option(k, v)
+        (dec.set_option if k in (0, 1, 2) else dec.debug_set)(k, v)
     per = N * K * 2 * (2 if op == 2 else 1)
     if copies <= 0:
         copies = max(2, int(np.ceil(400e6 / per)))           # ring of weights > 3x the 126 MB L2
@@ -38,20 +38,20 @@ def bench_gemm(M, N, K, op=0, reps=50, copies=0, warm=5, opts=()):
     W = S.normal((copies * N, K), 0, 2, 0.02, torch.bfloat16, DEV)
     W2 = S.normal((copies * N, K), 0, 3, 0.02, torch.bfloat16, DEV) if op == 2 else None
     out = torch.zeros(M, N, dtype=torch.bfloat16, device=DEV)
-    dec.set_option(3, 1)
-    dec.set_option(5, copies)
-    dec.set_option(4, warm)
+    dec.debug_set(3, 1)
+    dec.debug_set(5, copies)
+    dec.debug_set(4, warm)
     dec.op_linear(op, A, W[:N], W2[:N] if W2 is not None else None, out)
     torch.cuda.synchronize()
-    dec.set_option(4, reps)
+    dec.debug_set(4, reps)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     dec.op_linear(op, A, W[:N], W2[:N] if W2 is not None else None, out)
     e1.record()
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / reps
-    dec.set_option(3, 0)
-    dec.set_option(4, 1)
+    dec.debug_set(3, 0)
+    dec.debug_set(4, 1)
     dec.op_linear(0, A[:1], W[:N], None, out[:1])          # synchronising call: surfaces a device-side status
     dec.close()
     nw = 2 if op == 2 else 1
@@ -110,7 +110,7 @@ def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False, opts=
     dec = LSPDecoder(sh, w, SchedCfg(tau=wl.tau, delim_bitmap=S.delimiter_bitmap(sh.vocab, *wl.delim).to(DEV)), B, P + G,
                      device=DEV)
     for k, v in opts:
-        dec.set_option(k, v)
+        (dec.set_option if k in (0, 1, 2) else dec.debug_set)(k, v)
     tokens = torch.zeros(B, P + G, dtype=torch.int32, device=DEV)
     tokens[:, :P] = S.make_prompt(B, P, sh, 100).to(DEV)
 

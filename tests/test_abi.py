@@ -39,3 +39,14 @@ def test_sizes_and_argument_errors_without_gpu():
     h = ctypes.c_void_p()
     assert B.lib.lsp_init(ctypes.byref(h), None, None, None, None, None, 0, 1, 96, None) == -1
     assert B.lib.lsp_commit(None, None) == -1
+
+
+def test_internal_tuning_entry_is_exported_but_not_public():
+    """The tuning and benchmark knobs live behind lsp_debug_set, declared in the package's internal header only."""
+    from paper_2603_05454_b200 import build
+    l = ctypes.CDLL(build.build())
+    internal = open(os.path.join(ROOT, "paper_2603_05454_b200", "csrc", "lsp_tuning.h")).read()
+    assert re.search(r"\bint\s+lsp_debug_set\s*\(", internal) and hasattr(l, "lsp_debug_set")
+    assert "lsp_debug_set" not in _declared()
+    public = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "lsp.h")).read(), flags=re.S)
+    assert "tuning" not in public.lower()

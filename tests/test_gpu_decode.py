@@ -13,7 +13,8 @@ pytestmark = pytest.mark.gpu
 NEAR = oscan.FLAG_NEAR_THRESHOLD | oscan.FLAG_NEAR_TIE
 
 
-def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, max_steps=None, gains_seed=None):
+def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, max_steps=None, gains_seed=None,
+                    max_batch=1, extra_len=0, poison=False):
     """Runs the GPU path step by step, committing the ORACLE's lengths, and compares every step's outputs."""
     from paper_2603_05454_b200 import LSPDecoder
     tol = tol_for(shape.dtype)
@@ -39,13 +40,20 @@ def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, 
     sched.tie_tol = tol_z
     otok, orecs, (ock, ocv) = decode(om, prompt[0].numpy(), G, make_is_delim(*delim), oracle_policy(sched),
                                      score="pmax" if sched.score == 0 else "margin", max_steps=max_steps)
-    dec = LSPDecoder(shape, w_gpu, sched, 1, P + G, device=DEV)
+    dec = LSPDecoder(shape, w_gpu, sched, max_batch, P + G + extra_len, device=DEV)
+    if poison:
+        # NaN bit patterns in everything the caller hands over uninitialised: the whole cache and the staging planes
+        esz = 4 if shape.dtype == "fp32" else 2
+        pat, it = (0x7FC00000, torch.int32) if esz == 4 else (0x7FC0, torch.int16)
+        dec.kv_view().view(it).fill_(pat)
+        stage = shape.n_layers * 2 * max_batch * (P + G + extra_len) * shape.n_kv_heads * shape.head_dim * esz
+        dec.workspace[-((stage + 255) // 256 * 256):].view(it).fill_(pat)
     if impl is not None:
         dec.set_option(0, impl)
     if attn_impl is not None:
         dec.set_option(1, attn_impl)
         if attn_impl == 2:
-            dec.set_option(28, 0)          # the tcgen05 kernel at every row count, not only from its default threshold
+            dec.debug_set(28, 0)          # the tcgen05 kernel at every row count, not only from its default threshold
     tokens = torch.zeros(1, P + G, dtype=torch.int32, device=DEV)
     tokens[0, :P] = prompt[0].to(DEV)
     dec.begin(tokens, [P], [G])
@@ -84,7 +92,10 @@ def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, 
         kt = 4 * tol if shape.dtype == "bf16" else tol
         np.testing.assert_allclose(kv[l, 0, 0, :F], ock[l], atol=kt * max(1.0, np.abs(ock[l]).max()))
         np.testing.assert_allclose(kv[l, 1, 0, :F], ocv[l], atol=kt * max(1.0, np.abs(ocv[l]).max()))
-    assert not kv[:, :, 0, F:].any()          # nothing beyond the committed prefix was ever written
+    if poison:
+        assert np.isnan(kv[:, :, 0, F:]).all() and np.isnan(kv[:, :, 1:]).all()      # still the caller's bit pattern
+    else:
+        assert not kv[:, :, 0, F:].any()      # nothing beyond the committed prefix was ever written
     dec.close()
     return len(orecs), n_flagged
 
@@ -234,3 +245,46 @@ def test_bf16_model_with_learned_norm_gains():
     sh = S.ModelShape(3, 512, 4, 2, 128, 1024, 4096, dtype="bf16", head_scale=1.5, w_std=0.044)
     _teacher_forced(sh, 41, 40, 90, SchedCfg(tau=0.04), (1, 400), gains_seed=5)
     _teacher_forced(sh, 42, 200, 140, SchedCfg(mode=2, fixed_k=50), (1, 400), gains_seed=6, max_steps=3)
+
+
+@pytest.mark.parametrize("dtype,dh", [("bf16", 128), ("bf16", 64), ("fp32", 64)])
+def test_decode_does_not_read_memory_it_never_wrote(dtype, dh):
+    """The cache and the workspace arrive uninitialised (here: NaN bit patterns), the context is larger than the decode
+    (two sequence slots, max_len beyond prompt + generation) and neither the cache length nor the row count is a
+    multiple of the 128-key tile: a key tile's tail then covers rows nobody wrote, which must not reach any output."""
+    from paper_2603_05454_b200 import SchedCfg
+    hq, hkv = 4, 2
+    sh = S.ModelShape(2, hq * dh, hq, hkv, dh, 512, 2048, dtype=dtype, head_scale=1.5, w_std=0.5 / (hq * dh) ** 0.5)
+    _teacher_forced(sh, 51, 150, 170, SchedCfg(mode=2, fixed_k=45), (1, 200), max_steps=4, max_batch=2, extra_len=77,
+                    poison=True)
+
+
+def test_commit_lengths_survive_a_busy_stream():
+    """lsp_commit uploads the block lengths from a pinned mirror without waiting; with work queued ahead of it on the
+    stream the copy is still pending when the next lsp_denoise_step prepares its own descriptor.  The decode must be
+    the same as on an idle stream (no [MASK] left inside the committed prefix, same tokens, same records)."""
+    from paper_2603_05454_b200 import LSPDecoder, SchedCfg
+    sh = S.ModelShape(2, 512, 4, 2, 128, 1024, 4096, dtype="bf16", head_scale=1.5, w_std=0.044)
+    w = S.make_weights(sh, 5, device=DEV)
+    P, G, B = 24, 60, 2
+    prompt = S.make_prompt(B, P, sh, 6).to(DEV)
+    sched = SchedCfg(tau=0.04, delim_bitmap=S.delimiter_bitmap(sh.vocab, 1, 400).to(DEV))
+    big = torch.randn(4096, 4096, device=DEV)
+    runs = []
+    for busy in (False, True):
+        dec = LSPDecoder(sh, w, sched, B, P + G, device=DEV)
+        tokens = torch.full((B, P + G), sh.mask_id, dtype=torch.int32, device=DEV)
+        tokens[:, :P] = prompt
+        dec.begin(tokens, [P] * B, [G] * B)
+        recs = []
+        while dec.active()[1] > 0:
+            recs.append([(r["L_run"], r["L_commit"]) for r in dec.denoise_step()])
+            if busy:
+                for _ in range(12):              # about ten milliseconds of work ahead of the commit on the same stream
+                    big = (big @ big).clamp_(-1, 1)
+            dec.commit()                        # no synchronisation here: the next step starts with the copy still pending
+        tk = tokens.cpu().numpy().copy()
+        assert (tk != sh.mask_id).all(), "a committed position still holds [MASK]"
+        runs.append((tk, recs))
+        dec.close()
+    assert np.array_equal(runs[0][0], runs[1][0]) and runs[0][1] == runs[1][1]

@@ -65,7 +65,7 @@ def test_linear_bf16_weight_streaming_kernel(grid_mode, shape):
     M, N, K = shape
     tdt = torch.bfloat16
     dec = _dec("bf16")
-    dec.set_option(17, grid_mode)
+    dec.debug_set(17, grid_mode)
     A = S.normal((M, K), 2, 1, 1.0, tdt, DEV)
     W = S.normal((N, K), 2, 2, 0.05, tdt, DEV)
     W2 = S.normal((N, K), 2, 3, 0.05, tdt, DEV)
@@ -108,7 +108,7 @@ def test_linear_bf16_cluster_split_of_two_row_tiles(case):
     tdt = torch.bfloat16
     dec = _dec("bf16")
     for k, v in opts.items():
-        dec.set_option(k, v)
+        dec.debug_set(k, v)
     A = S.normal((M, K), 3, 1, 1.0, tdt, DEV)
     W = S.normal((N, K), 3, 2, 0.05, tdt, DEV)
     W2 = S.normal((N, K), 3, 3, 0.05, tdt, DEV)
@@ -156,7 +156,7 @@ def test_linear_bf16_seeded_random_shapes_and_kernel_options():
             if rng.random() < p:
                 opts[key] = rng.choice(vals)
         for k, v in {**defaults, **opts}.items():
-            dec.set_option(k, v)
+            dec.debug_set(k, v)
         A = S.normal((M, K), done, 1, 1.0, torch.bfloat16, DEV)
         W = S.normal((N, K), done, 2, 0.05, torch.bfloat16, DEV)
         W2 = S.normal((N, K), done, 3, 0.05, torch.bfloat16, DEV)

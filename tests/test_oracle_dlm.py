@@ -163,3 +163,14 @@ def test_fp32_mode_rounds_nothing():
     ck, cv = m.empty_cache()
     x = np.random.default_rng(1).normal(size=(3, 7))
     assert m.r(x) is x
+
+
+def test_one_layer_at_a_time_mode_is_the_same_arithmetic():
+    sh = _tiny(dtype="bf16")
+    w = S.make_weights(sh, 3)
+    a, b = dlm.OracleDLM(sh, w), dlm.OracleDLM(sh, w, one_layer_at_a_time=True)
+    ids, pos = np.array([5, 9, 49, 49]), np.arange(4) + 3
+    ck, cv = a.empty_cache()
+    la, ka, va = a.forward(ids, pos, ck, cv, [2, 3])
+    lb, kb, vb = b.forward(ids, pos, ck, cv, [2, 3])
+    assert np.array_equal(la, lb) and all(np.array_equal(x, y) for x, y in zip(ka + va, kb + vb))
