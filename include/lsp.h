@@ -130,7 +130,12 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
 /* Implementation switches: key 0 = GEMM implementation for bf16 models (0 = CUDA-core reference kernels, 1 = tcgen05,
  * default 1); key 1 = attention implementation for bf16 models (0 = CUDA-core, 1 = mma.sync tensor cores, 2 = default:
  * tcgen05 tensor cores for head_dim 128, else as 1); key 2 = per-class CUDA-event timing (0 off, 1 on; see
- * lsp_last_timing).  Any other key: LSP_ERR_ARG. */
+ * lsp_last_timing); key 3 = K/V layout of a pass: 0 (default, the contract) = the pass writes its keys / values to
+ * staging planes and lsp_commit appends the pending block's rows to the cache as one contiguous copy per layer
+ * (Algorithm 1, AppendToCache); 1 = in place: the pass writes every row's K/V at that row's absolute position in the
+ * cache buffer, behind the committed prefix, so the append is only the length bump (rows [F, F + rows) of a sequence
+ * then hold provisional values between steps; rows [0, F) are final and never rewritten in either layout).  The layout
+ * cannot change in the middle of a decode (LSP_ERR_STATE).  Any other key: LSP_ERR_ARG. */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(128) k_attn_mma(const bf16* __restrict__ q, co
                                                   const bf16* __restrict__ cache_v, const bf16* __restrict__ stage_k,
                                                   const bf16* __restrict__ stage_v, bf16* __restrict__ out, StepDesc sd,
                                                   int n_heads, int n_kv_heads, size_t cache_seq_elems,
-                                                  float scale_log2) {
+                                                  float scale_log2, int inplace) {
   constexpr int LD = DH + 8;            // padded row (elements): 16-byte shift per row, conflict-free ldmatrix
   constexpr int CPR = DH / 8;           // 16-byte chunks per row
   extern __shared__ __align__(16) uint8_t attn_smem[];
@@ -69,8 +69,8 @@ __global__ void __launch_bounds__(128) k_attn_mma(const bf16* __restrict__ q, co
   const int rows_total = Qn * G;
   const int row_base = blockIdx.x * AM_BM;
   if (row_base >= rows_total) return;
-  const int F = sd.F[b];
-  const int S = F + Qn;
+  const int S = sd.F[b] + Qn;
+  const int F = inplace ? S : sd.F[b];      // in-place layout: this pass's K/V rows already sit behind the prefix in the cache
   const int ldq = n_heads * DH, ldkv = n_kv_heads * DH;
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
   const bf16* ck = cache_k + (size_t)b * cache_seq_elems + kvh * DH;

@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(128) k_attn_simt(const T* __restrict__ q, cons
                                                    const T* __restrict__ cache_v, const T* __restrict__ stage_k,
                                                    const T* __restrict__ stage_v, T* __restrict__ out, StepDesc sd,
                                                    int n_heads, int n_kv_heads, size_t cache_seq_elems,
-                                                   float scale) {
+                                                   float scale, int inplace) {
   __shared__ float Qs[AS_BQ][DH];
   __shared__ float Ks[AS_BK][DH + 1];
   __shared__ float Vs[AS_BK][DH];
@@ -27,8 +27,8 @@ __global__ void __launch_bounds__(128) k_attn_simt(const T* __restrict__ q, cons
   const int Qn = sd.row_off[b + 1] - r0;
   const int q0 = blockIdx.x * AS_BQ;
   if (q0 >= Qn) return;
-  const int F = sd.F[b];
-  const int S = F + Qn;
+  const int S = sd.F[b] + Qn;
+  const int F = inplace ? S : sd.F[b];      // in-place layout: this pass's K/V rows already sit behind the prefix in the cache
   const int kvh = h / (n_heads / n_kv_heads);
   const int ldq = n_heads * DH, ldkv = n_kv_heads * DH;
   const int t = threadIdx.x, lane = t & 31, w = t >> 5;

@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(AU_THREADS, 1)
 k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ CUtensorMap map_cv,
             const __grid_constant__ CUtensorMap map_sk, const __grid_constant__ CUtensorMap map_sv,
             const bf16* __restrict__ q, bf16* __restrict__ out, StepDesc sd, int n_heads, int n_kv_heads, int max_len,
-            float scale_log2, int cluster, unsigned* status) {
+            float scale_log2, int cluster, int inplace, unsigned* status) {
   constexpr int DH = 128;
   extern __shared__ uint8_t smem_raw[];
   pdl_release();
@@ -127,8 +127,9 @@ k_attn_umma(const __grid_constant__ CUtensorMap map_ck, const __grid_constant__ 
   const int C = cluster > 1 ? cluster : 1;
   const int rank = (int)(blockIdx.x % C);
   const int row_base = (int)(blockIdx.x / C) * AU_BM;
-  const int F = sd.F[b];
-  const int n_c = (F + AU_BN - 1) / AU_BN, n_s = (Qn + AU_BN - 1) / AU_BN;
+  // in-place layout: this pass's K/V rows already sit behind the prefix in the cache, so every key tile is a cache tile
+  const int F = sd.F[b] + (inplace ? Qn : 0);
+  const int n_c = (F + AU_BN - 1) / AU_BN, n_s = inplace ? 0 : (Qn + AU_BN - 1) / AU_BN;
   const int n_all = (row_base < rows_total) ? n_c + n_s : 0;       // a CTA past the last row does nothing
   const int n_tiles = n_all > rank ? (n_all - rank + C - 1) / C : 0;   // this CTA's tiles; t below counts them
   const int ldq = n_heads * DH;

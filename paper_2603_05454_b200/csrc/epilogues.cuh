@@ -67,6 +67,13 @@ struct EpiQKVRope {
   const float2* cs; // [max_len, dh/2] (cos, sin)
   const int* row_pos;
   int n_heads, n_kv_heads, half; // half = dh / 2
+  // K/V destination row of packed row m: m itself (staging planes), or, with seq_stride > 0, the row's own cache slot
+  // row_seq[m] * seq_stride + row_pos[m] (k_stage / v_stage then point at the cache planes: the in-place layout)
+  const int* row_seq = nullptr;
+  int seq_stride = 0;
+  __device__ __forceinline__ size_t kv_row(int m) const {
+    return seq_stride > 0 ? (size_t)row_seq[m] * seq_stride + row_pos[m] : (size_t)m;
+  }
   __device__ __forceinline__ int row0(int j) const { return (j / half) * 2 * half + (j % half); }
   __device__ __forceinline__ int row1(int j) const { return row0(j) + half; }
   __device__ __forceinline__ void elem(int m, int j, float a0, float a1) const {
@@ -77,11 +84,11 @@ struct EpiQKVRope {
       const float r0 = a0 * c.x - a1 * c.y;
       const float r1 = a1 * c.x + a0 * c.y;
       T* dst = (h < n_heads) ? q_out + (size_t)m * n_heads * dh + h * dh
-                             : k_stage + (size_t)m * n_kv_heads * dh + (h - n_heads) * dh;
+                             : k_stage + kv_row(m) * n_kv_heads * dh + (h - n_heads) * dh;
       dst[i] = from_f<T>(r0);
       dst[i + half] = from_f<T>(r1);
     } else {
-      T* dst = v_stage + (size_t)m * n_kv_heads * dh + (h - n_heads - n_kv_heads) * dh;
+      T* dst = v_stage + kv_row(m) * n_kv_heads * dh + (h - n_heads - n_kv_heads) * dh;
       dst[i] = from_f<T>(a0);
       dst[i + half] = from_f<T>(a1);
     }

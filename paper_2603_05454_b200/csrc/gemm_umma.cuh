@@ -204,11 +204,11 @@ __device__ __forceinline__ void epi16(const EpiQKVRope<bf16>& e, int m, int j, c
       r1[2 * q + 1] = a1[2 * q + 1] * c.z + a0[2 * q + 1] * c.w;
     }
     dst = (h < e.n_heads) ? e.q_out + (size_t)m * e.n_heads * dh + h * dh
-                          : e.k_stage + (size_t)m * e.n_kv_heads * dh + (h - e.n_heads) * dh;
+                          : e.k_stage + e.kv_row(m) * e.n_kv_heads * dh + (h - e.n_heads) * dh;
   } else {
 #pragma unroll
     for (int q = 0; q < 16; ++q) { r0[q] = a0[q]; r1[q] = a1[q]; }
-    dst = e.v_stage + (size_t)m * e.n_kv_heads * dh + (h - e.n_heads - e.n_kv_heads) * dh;
+    dst = e.v_stage + e.kv_row(m) * e.n_kv_heads * dh + (h - e.n_heads - e.n_kv_heads) * dh;
   }
   uint4* p0 = reinterpret_cast<uint4*>(dst + i);
   uint4* p1 = reinterpret_cast<uint4*>(dst + i + e.half);

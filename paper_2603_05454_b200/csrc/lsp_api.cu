@@ -61,6 +61,7 @@ struct lsp_ctx {
   bool proposed = false;
   int score_rows = 0;
   int last_M = 0;
+  int kv_inplace = 0;               // K/V layout: 0 = staging planes + append copy, 1 = written in place (see lsp_set_option key 3)
   int last_attn_kernel = 0, last_attn_cluster = 1;   // what the last attention launch was (see lsp_get_counters)
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   float timing_ms[8] = {0};
@@ -308,7 +309,7 @@ int check_status(lsp_ctx* c) {
 // of the pass's own rows).  Reads the uploaded descriptor (F, row_off), Q from q, K/V from the cache and the staging
 // planes of layer l; writes out.  max_q: most query rows of one sequence; max_keys: most keys of one sequence.
 template <typename T>
-int run_attention(lsp_ctx* c, int l, const T* Qb, T* Att, int B, int maxQ, int max_keys) {
+int run_attention(lsp_ctx* c, int l, const T* Qb, T* Att, int B, int maxQ, int max_keys, int inplace) {
   const lsp_model_cfg& m = c->m;
   const StepDesc sd = desc_of(c);
   const int dh = m.head_dim, kvd = m.n_kv_heads * dh;
@@ -343,7 +344,7 @@ int run_attention(lsp_ctx* c, int l, const T* Qb, T* Att, int B, int maxQ, int m
       const float sl2 = scale * 1.4426950408889634f;
       const CUtensorMap* mp = &c->attn_maps[4 * l];
       launch_k(c->pdl, k_attn_umma, g3, dim3(AU_THREADS), (size_t)AU_SMEM, c->stream, cl, mp[0], mp[1], mp[2], mp[3],
-               (const bf16*)Qb, Att, sd, m.n_heads, m.n_kv_heads, c->max_len, sl2, cl, c->d_status);
+               (const bf16*)Qb, Att, sd, m.n_heads, m.n_kv_heads, c->max_len, sl2, cl, inplace, c->d_status);
       c->last_attn_kernel = 2;
       c->last_attn_cluster = cl;
       done = true;
@@ -356,9 +357,9 @@ int run_attention(lsp_ctx* c, int l, const T* Qb, T* Att, int B, int maxQ, int m
       dim3 g2((maxQ * G + AM_BM - 1) / AM_BM, m.n_kv_heads, B);
       const float sl2 = scale * 1.4426950408889634f;
       if (dh == 128)
-        launch_k(c->pdl, k_attn_mma<128>, dim3(g2), dim3(128), attn_mma_smem_bytes<128>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
+        launch_k(c->pdl, k_attn_mma<128>, dim3(g2), dim3(128), attn_mma_smem_bytes<128>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2, inplace);
       else
-        launch_k(c->pdl, k_attn_mma<64>, dim3(g2), dim3(128), attn_mma_smem_bytes<64>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2);
+        launch_k(c->pdl, k_attn_mma<64>, dim3(g2), dim3(128), attn_mma_smem_bytes<64>(), c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads, (size_t)c->max_len * kvd, sl2, inplace);
       c->last_attn_kernel = 1;
       done = true;
     }
@@ -367,10 +368,10 @@ int run_attention(lsp_ctx* c, int l, const T* Qb, T* Att, int B, int maxQ, int m
   if (done) {
   } else if (dh == 128)
     launch_k(c->pdl, k_attn_simt<T, 128>, dim3(grid), dim3(128), 0, c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
-                                                     (size_t)c->max_len * kvd, scale);
+                                                     (size_t)c->max_len * kvd, scale, inplace);
   else
     launch_k(c->pdl, k_attn_simt<T, 64>, dim3(grid), dim3(128), 0, c->stream, Qb, cK, cV, stK, stV, Att, sd, m.n_heads, m.n_kv_heads,
-                                                    (size_t)c->max_len * kvd, scale);
+                                                    (size_t)c->max_len * kvd, scale, inplace);
   seg_end(c);
   CU(cudaGetLastError());
   return LSP_OK;
@@ -426,16 +427,19 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   seg_end(c);
   count_launch(c, CLS_MISC);
   const size_t plane = (size_t)c->max_rows * kvd;           // elements per staged (layer, K|V) plane
+  const size_t cplane = (size_t)c->max_batch * c->max_len * kvd;
   for (int l = 0; l < m.n_layers; ++l) {
-    T* stK = (T*)c->stage + (size_t)(2 * l) * plane;
-    T* stV = stK + plane;
+    // this pass's K/V: the staging planes, or (in-place layout) each row's own slot in the cache planes
+    T* stK = c->kv_inplace ? (T*)c->kv_cache + (size_t)(2 * l) * cplane : (T*)c->stage + (size_t)(2 * l) * plane;
+    T* stV = stK + (c->kv_inplace ? cplane : plane);
     seg_begin(c, CLS_MISC);
     launch_k(c->pdl, k_rmsnorm<T>, dim3(M), dim3(256), 0, c->stream, X, (const T*)c->attn_norm[l], Nrm, nullptr, d, m.rms_eps);
     seg_end(c);
     count_launch(c, CLS_MISC);
     CU(cudaGetLastError());
     {
-      EpiQKVRope<T> e{Qb, stK, stV, c->rope_cs, c->row_pos, m.n_heads, m.n_kv_heads, dh / 2};
+      EpiQKVRope<T> e{Qb, stK, stV, c->rope_cs, c->row_pos, m.n_heads, m.n_kv_heads, dh / 2, c->row_seq,
+                      c->kv_inplace ? c->max_len : 0};
       const int rc = run_gemm<T>(c, Nrm, (const T*)c->w_qkv[l], (const T*)c->w_qkv[l], M, (qd + 2 * kvd) / 2, d,
                                  qd + 2 * kvd, e);
       if (rc) return rc;
@@ -451,7 +455,7 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
       int max_keys = 0;
       for (int b = 0; b < B; ++b)
         if (c->N[b] > 0) max_keys = std::max(max_keys, c->F[b] + c->pend[b] + (scattered ? c->G[b] : c->N[b]));
-      const int rc = run_attention<T>(c, l, Qb, Att, B, maxQ, max_keys);
+      const int rc = run_attention<T>(c, l, Qb, Att, B, maxQ, max_keys, c->kv_inplace);
       if (rc) return rc;
     }
     {
@@ -709,6 +713,15 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
   if (key == 0) c->gemm_impl = value;
   else if (key == 1) c->attn_impl = value;
   else if (key == 2) c->timing = value;
+  else if (key == 3) {
+    if (c->tokens && c->step > 0) {
+      bool active = false;
+      for (int b = 0; b < c->batch; ++b) active |= c->N[b] > 0;
+      if (active && (value != 0) != (c->kv_inplace != 0))
+        return fail(c, LSP_ERR_STATE, "lsp_set_option: the K/V layout cannot change in the middle of a decode");
+    }
+    c->kv_inplace = value ? 1 : 0;
+  }
   else return fail(c, LSP_ERR_ARG, "lsp_set_option: unknown key %d", key);
   return LSP_OK;
 }
@@ -813,10 +826,12 @@ int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
   dim3 grid(chunks, m.n_layers * 2, B);
   seg_begin(c, CLS_COMMIT);
   const bool scattered = c->s.topology == 1;
-  if (!scattered || max_pend > 0) {
+  const bool copy = !c->kv_inplace;          // in-place layout: the pending block's K/V are already where they belong
+  if (!copy) grid = dim3(1, 1, B);
+  if ((!scattered || max_pend > 0) && (copy || !scattered)) {
     launch_k(c->pdl, k_commit_append, dim3(grid), dim3(256), 0, c->stream, desc_of(c), (const uint4*)c->stage, (uint4*)c->kv_cache,
                                                  stage_plane_v4, cache_plane_v4, cache_seq_v4, row_v4, c->yhat,
-                                                 c->tokens, c->tok_stride, scattered ? 0 : 1);
+                                                 c->tokens, c->tok_stride, scattered ? 0 : 1, copy ? 1 : 0);
     count_launch(c, CLS_COMMIT);
   }
   if (scattered) {
@@ -830,7 +845,7 @@ int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
   }
   seg_end(c);
   for (int b = 0; b < B; ++b)
-    if (c->N[b] > 0) c->counters[CNT_APPEND_BYTES] += 2.0 * c->pend[b] * kvd * c->esz * 2.0 * m.n_layers;
+    if (c->N[b] > 0 && copy) c->counters[CNT_APPEND_BYTES] += 2.0 * c->pend[b] * kvd * c->esz * 2.0 * m.n_layers;
   CU(cudaGetLastError());
   for (int b = 0; b < B; ++b) {
     if (c->N[b] == 0) continue;
@@ -992,8 +1007,8 @@ int lsp_op_attention(lsp_ctx* c, int layer, const void* q, const void* k_new, co
   char* stK = c->stage + (size_t)(2 * layer) * plane;
   CU(cudaMemcpyAsync(stK, k_new, (size_t)M * kvd * c->esz, cudaMemcpyDeviceToDevice, c->stream));
   CU(cudaMemcpyAsync(stK + plane, v_new, (size_t)M * kvd * c->esz, cudaMemcpyDeviceToDevice, c->stream));
-  const int rc = c->m.dtype == 0 ? run_attention<float>(c, layer, (const float*)q, (float*)out, batch, maxQ, max_keys)
-                                 : run_attention<bf16>(c, layer, (const bf16*)q, (bf16*)out, batch, maxQ, max_keys);
+  const int rc = c->m.dtype == 0 ? run_attention<float>(c, layer, (const float*)q, (float*)out, batch, maxQ, max_keys, 0)
+                                 : run_attention<bf16>(c, layer, (const bf16*)q, (bf16*)out, batch, maxQ, max_keys, 0);
   if (rc) return rc;
   CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
   CU(cudaStreamSynchronize(c->stream));

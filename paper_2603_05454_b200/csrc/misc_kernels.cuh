@@ -284,12 +284,12 @@ __global__ void k_commit_append(StepDesc sd, const uint4* __restrict__ stage, ui
                                 size_t cache_seq_v4,     // uint4 per sequence inside a cache plane
                                 int row_v4,              // uint4 per row (n_kv_heads * head_dim * sizeof(T) / 16)
                                 const int32_t* __restrict__ yhat, int32_t* __restrict__ tokens, int tok_stride,
-                                int write_tokens) {
+                                int write_tokens, int copy_rows) {
   pdl_begin();
   const int b = blockIdx.z;
   const int plane = blockIdx.y;
   const int pend = sd.pend[b];
-  const size_t n = (size_t)pend * row_v4;
+  const size_t n = copy_rows ? (size_t)pend * row_v4 : 0;      // in-place layout: nothing to move, the append is the length bump
   const uint4* src = stage + plane * stage_plane_v4 + (size_t)sd.row_off[b] * row_v4;
   uint4* dst = cache + plane * cache_plane_v4 + b * cache_seq_v4 + (size_t)sd.F[b] * row_v4;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
