@@ -9,8 +9,11 @@ CUDA device is present the generator produces the weights there (same bits as on
 over one layer at a time; all of the oracle's arithmetic runs on the host in float64.
 
 Every stored block is one (policy, pass): the step's N, rows, L', L, flags, tau, then yhat, p_max and delta of every
-masked position.  The header carries a hash of the oracle's and the generator's sources; the test recomputes the
-records itself when that hash no longer matches.
+masked position.  The block "exact" is pass 0 once more with NO activation rounding (the same bf16 weights, float64
+throughout): the distance between it and the bf16-rounding oracle is what rounding to bf16 at the declared points does
+to the scores at this depth, i.e. the yardstick for how far two correct bf16 pipelines may sit from each other.
+The header carries a hash of the oracle's and the generator's sources; the test recomputes the records itself when
+that hash no longer matches.
 """
 import argparse
 import hashlib
@@ -87,6 +90,19 @@ def compute(name, log=print):
         out[pname] = recs
         log(f"{name}/{pname}: {len(recs)} passes in {time.time() - t0:.0f} s; rows {[r['rows'] for r in recs]}, "
             f"L {[r['L_commit'] for r in recs]}")
+    # pass 0 without any activation rounding (policy-independent)
+    import dataclasses
+    from oracle.scores import scores_from_logits
+    t0 = time.time()
+    om_x = dlm.OracleDLM(dataclasses.replace(sh, dtype="fp32"), w, one_layer_at_a_time=True)
+    P, G = wl.prompt_len, wl.gen_len
+    ids = np.concatenate([prompt, np.full(G, sh.mask_id)])
+    ck, cv = om_x.empty_cache()
+    logits, _, _ = om_x.forward(ids, np.arange(P + G), ck, cv, np.arange(P, P + G))
+    yhat, pmax, delta = scores_from_logits(logits, sh.mask_id)
+    out["exact"] = [dict(step=0, n_before=G, rows=P + G, L_run=0, L_commit=0, flags=0, tau_used=float("nan"), yhat=yhat,
+                         pmax=pmax, delta=delta)]
+    log(f"{name}/exact: pass 0 without rounding in {time.time() - t0:.0f} s")
     return out
 
 

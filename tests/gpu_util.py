@@ -15,25 +15,27 @@ def tol_for(dtype):
 
 
 def tol_logit(dtype, z_rms, n_layers=1):
-    """Tolerance on logit-scale quantities (logits, the margin delta) for logits of RMS magnitude z_rms.
+    """Tolerance on logit-scale quantities (logits, the margin delta) for logits of RMS magnitude z_rms, for the shallow
+    models (1-3 layers) the step-by-step decode tests run.  (At full depth the bound is not a formula: the oracle
+    measures its own bf16 rounding noise, see test_gpu_fulldepth.py.)
 
-    fp32: 1e-4 relative to the logit scale.
-    bf16: two correct bf16 pipelines agree only to about one bf16 ulp (2^-8 relative) per element at every point
-    where an activation is rounded, because a last-bit difference in fp32 summation order flips roundings and the
-    flips spread to every later element.  The model has about 6 rounding points per layer (norm, Q/K/V, attention
-    probabilities and output, two residual updates, SwiGLU product), their effects add like a random walk, and the
-    comparison takes the maximum over ~1e4-1e5 (row, column) pairs (about 4.5 sigma):
-        tol = 2^-8 * 4.5 * sqrt(6 * n_layers) * z_rms,   never below 2e-2."""
+    fp32: 1e-4 relative to the logit scale (measured: at most 6e-6 z_rms).
+    bf16: two correct bf16 pipelines agree only to about one bf16 ulp (2^-8 relative) per element at every point where
+    an activation is rounded, because a last-bit difference in fp32 summation order flips roundings and the flips spread
+    to every later element.  About 6 rounding points per layer, adding like a random walk, maximum over ~1e4-1e5
+    (row, column) pairs (about 4.5 sigma):
+        tol = 2^-8 * 4.5 * sqrt(6 * n_layers) * z_rms,   never below 2e-2.
+    Measured on B200 over all decode tests (printed per test, pytest -s): at most 55 % of this allowance is used
+    (0.034 z_rms at two layers, 0.022 z_rms on a full-width single layer)."""
     if dtype == "fp32":
         return 1e-4 * max(1.0, z_rms)
     return max(2e-2, 2.0 ** -8 * 4.5 * (6.0 * max(1, n_layers)) ** 0.5 * z_rms)
 
 
-def tol_prob(dtype, tol_z):
-    """Tolerance on p_max given the logit tolerance tol_z of the same model: p_max = softmax(z)_max, so
-    |dp| = p (1 - p) |dz_max - sum_j w_j dz_j| <= |dz| / 4 with dz the error of the top logit against the softmax-
-    weighted mean of the others' errors (which averages down).  Never below the fixed probability tolerance."""
-    return max(tol_for(dtype), 0.25 * tol_z) if dtype != "fp32" else tol_for(dtype)
+def tol_prob(dtype, tol_z=None):
+    """Tolerance on p_max: the benchmark's 2e-2 absolute for bf16 models, 1e-4 for fp32, as stated; no widening with the
+    logit scale (measured maximum over the 1-3-layer decode tests on B200: 1.8e-2 for bf16, 1e-6 for fp32)."""
+    return tol_for(dtype)
 
 
 def make_pair(shape, seed):
@@ -48,3 +50,14 @@ def oracle_policy(s, flag_tol=None):
     return dict(mode=s.mode, tau=float(np.float32(s.tau)), alpha=float(np.float32(s.alpha)),
                 beta=float(np.float32(s.beta)), l_min=s.l_min, W=s.snap_window, fixed_k=s.fixed_k,
                 flag_tol=float(np.float32(s.flag_tol)), tie_tol=float(np.float32(s.tie_tol)))
+
+
+def report_parity(line):
+    """Measured error against its allowance, printed (pytest -s) and appended to $LSP_PARITY_REPORT/decode.txt."""
+    import os
+    print(line)
+    d = os.environ.get("LSP_PARITY_REPORT")
+    if d:
+        os.makedirs(d, exist_ok=True)
+        with open(os.path.join(d, "decode.txt"), "a") as f:
+            f.write(line + "\n")

@@ -7,7 +7,7 @@ import torch
 import lsp_synth as S
 from oracle import scan as oscan
 from oracle.decode import decode, make_is_delim
-from gpu_util import tol_prob, DEV, make_pair, oracle_policy, tol_for, tol_logit
+from gpu_util import tol_prob, DEV, make_pair, oracle_policy, report_parity, tol_for, tol_logit
 
 pytestmark = pytest.mark.gpu
 NEAR = oscan.FLAG_NEAR_THRESHOLD | oscan.FLAG_NEAR_TIE
@@ -61,10 +61,12 @@ def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, 
     dec.begin(tokens, [P], [G])
     n_flagged = 0
     snap_prefix = None
+    used_p = used_z = 0.0
     for o in orecs:
         rec = dec.denoise_step()[0]
         y, p, m = dec.scores()
         assert rec["n_before"] == o["n_before"] and rec["rows"] == o["rows"]
+        used_p, used_z = max(used_p, float(np.abs(p - o["pmax"]).max())), max(used_z, float(np.abs(m - o["delta"]).max()))
         assert np.abs(p - o["pmax"]).max() <= tol_p, (o["step"], np.abs(p - o["pmax"]).max(), tol_p)
         assert np.abs(m - o["delta"]).max() <= tol_z, (o["step"], np.abs(m - o["delta"]).max(), tol_z)
         diff = np.nonzero(y != o["yhat"])[0]
@@ -101,6 +103,9 @@ def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, 
     else:
         assert not kv[:, :, 0, F:].any()      # nothing beyond the committed prefix was ever written
     dec.close()
+    report_parity(f"{shape.dtype} L={shape.n_layers} d={shape.d_model} heads {shape.n_heads}/{shape.n_kv_heads}x{shape.head_dim} "
+                  f"ffn {shape.d_ffn} V={shape.vocab} P={P} G={G} steps {len(orecs)}: z_rms {zr[0]:.2f}; max|dp_max| {used_p:.2e} "
+                  f"of {tol_p:.2e} allowed; max|ddelta| {used_z:.2e} of {tol_z:.2e} allowed; flagged steps {n_flagged}")
     return len(orecs), n_flagged
 
 
