@@ -15,7 +15,10 @@ Prints ONE JSON line:
                  with per-launch CUDA events in a second pass over the same K decodes
   classes        the same figures for every kernel class (attention, LM head, append, ...)
   cpu_baseline   the CPU oracle timed on a bounded sample of the same workload (rank 0, N = 1 only)
-  also           a shorter run of the Dream-7B-shaped decode (cfg4), whose passes are tensor-bound
+  also           the other workloads: a shorter run of the Dream-7B-shaped decode (cfg4, tensor-bound passes), the
+                 head-only configuration (cfg2) and the long batched decode next to scattered acceptance (cfg5)
+  loop_variants  ms per pass of the same decode with the block lengths kept on the device and / or the in-place K/V
+                 layout, beside the synchronous loop with the append copy (the contract, which `value` times)
   adaptive_tau   the same workload decoded in the adaptive-threshold mode (Eq. 2, block in [0.25 N, 0.50 N]): passes,
                  suffix length per pass (geometric decay), rows touched in total against the G/beta..G/alpha bounds
 
@@ -338,7 +341,8 @@ def run_adaptive_leg(dec, wl, bm, tokens, Pl, Gl, steps, barrier):
     return out
 
 
-def run_decode_bench(wl, dev, rank, world, peaks, steps, warmup, sampler=None, with_e2e=True, adaptive=False):
+def run_decode_bench(wl, dev, rank, world, peaks, steps, warmup, sampler=None, with_e2e=True, adaptive=False,
+                     variants=False):
     import numpy as np
     import torch
     import lsp_synth as S
@@ -399,6 +403,33 @@ def run_decode_bench(wl, dev, rank, world, peaks, steps, warmup, sampler=None, w
         res["h2d"] = host_in.numel() * 4
         res["d2h"] = host_out.numel() * 4
         assert int((host_out == sh.mask_id).sum()) == 0 and bool((host_out[:, :P] == host_in[:, :P]).all())
+
+    # Section 8(f)4-style variants of the loop on the same resident decoder: block lengths kept on the device (the host
+    # enqueues pass k+1 before it has read L_k) and the in-place K/V layout (the append degenerates to a length bump).
+    # The synchronous loop with the staged layout and the append copy (timed above) stays the contract.
+    if variants:
+        res["variants"] = {"sync_staged": {"ms_per_pass": ms / passes, "tokens_per_s": B * G * steps / (ms * 1e-3),
+                                           "kv_append_bytes_per_token": cnt["append_bytes"] / max(1.0, cnt["tokens"])}}
+        for vname, (lag, inpl) in (("lagged_staged", (1, 0)), ("sync_inplace", (0, 1)), ("lagged_inplace", (1, 1))):
+            dec.set_option(4, lag)
+            dec.set_option(3, inpl)
+            decode_resident()
+            dec.reset_counters()
+            barrier()
+            ev0.record()
+            p2 = 0
+            for _ in range(steps):
+                p2 += decode_resident()
+            ev1.record()
+            barrier()
+            assert int((tokens == sh.mask_id).sum()) == 0, "decode left masked positions"
+            c2 = dec.counters()
+            v_ms = ev0.elapsed_time(ev1)
+            res["variants"][vname] = {"ms_per_pass": v_ms / p2, "tokens_per_s": B * G * steps / (v_ms * 1e-3),
+                                      "passes_per_decode": p2 / steps,
+                                      "kv_append_bytes_per_token": c2["append_bytes"] / max(1.0, c2["tokens"])}
+        dec.set_option(4, 0)
+        dec.set_option(3, 0)
 
     # second pass over the same decodes with one CUDA-event pair around every launch (per-class kernel time)
     dec.set_option(2, 1)
@@ -649,7 +680,8 @@ def main():
     if args.workload == "cfg5":
         print(json.dumps(topology_line(wl, dev, peaks, peak_kind, args.warmup, sampler)))
         return 0
-    r = run_decode_bench(wl, dev, rank, world, peaks, args.steps, args.warmup, sampler, adaptive=(world == 1))
+    r = run_decode_bench(wl, dev, rank, world, peaks, args.steps, args.warmup, sampler, adaptive=(world == 1),
+                         variants=(world == 1))
     (ms_max, e2e_max), tokens_total = reduce_replicas([r["ms"], r.get("e2e_ms", 0.0)], r["tokens"], world, dev)
     value = tokens_total / (ms_max * 1e-3)
     gemm = r["classes"]["gemm"]
@@ -680,6 +712,8 @@ def main():
             "gpu_launches": r["launches"], "clocks": r["clocks"]}
     if r.get("adaptive"):
         line["adaptive_tau"] = r["adaptive"]
+    if r.get("variants"):
+        line["loop_variants"] = r["variants"]
     if r.get("gemm_chain"):
         gc = r["gemm_chain"]
         line["roofline"]["back_to_back"] = {

@@ -135,7 +135,13 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * (Algorithm 1, AppendToCache); 1 = in place: the pass writes every row's K/V at that row's absolute position in the
  * cache buffer, behind the committed prefix, so the append is only the length bump (rows [F, F + rows) of a sequence
  * then hold provisional values between steps; rows [0, F) are final and never rewritten in either layout).  The layout
- * cannot change in the middle of a decode (LSP_ERR_STATE).  Any other key: LSP_ERR_ARG. */
+ * cannot change in the middle of a decode (LSP_ERR_STATE); key 4 = where lsp_generate keeps the block lengths: 0
+ * (default) = it reads L back after every pass before it enqueues the next; 1 = device-resident: the scan's L feeds the
+ * commit kernel directly, the next pass's descriptor is derived from it on the device, and the host enqueues pass k+1
+ * while pass k runs, reading L one step late (it sizes launches from row counts it knows a step late, upper bounds for
+ * the LM-head rows; rows beyond the real ones are inert).  Same tokens, boundaries and records either way; prefix
+ * topology only, and only while per-class timing is off (otherwise the synchronous loop runs).  Any other key:
+ * LSP_ERR_ARG. */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
 
 /* Algorithm 1, state initialisation: X_F <- prompt, X_A <- masks, K <- empty.  tokens: device int32

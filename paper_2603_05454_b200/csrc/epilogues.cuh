@@ -79,6 +79,7 @@ struct EpiQKVRope {
   __device__ __forceinline__ void elem(int m, int j, float a0, float a1) const {
     const int h = j / half, i = j % half;
     const int dh = 2 * half;
+    if (h >= n_heads && seq_stride > 0 && row_seq[m] < 0) return;      // in-place layout: a row of no sequence has no cache slot
     if (h < n_heads + n_kv_heads) {
       const float2 c = cs[(size_t)row_pos[m] * half + i];
       const float r0 = a0 * c.x - a1 * c.y;

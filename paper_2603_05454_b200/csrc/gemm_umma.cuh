@@ -193,6 +193,7 @@ __device__ __forceinline__ void epi16(const EpiQKVRope<bf16>& e, int m, int j, c
   const int dh = 2 * e.half;
   float r0[16], r1[16];
   bf16* dst;
+  if (h >= e.n_heads && e.seq_stride > 0 && e.row_seq[m] < 0) return;      // in-place layout: a row of no sequence has no cache slot
   if (h < e.n_heads + e.n_kv_heads) {
     const float4* c4 = reinterpret_cast<const float4*>(e.cs + (size_t)e.row_pos[m] * e.half + i);
 #pragma unroll

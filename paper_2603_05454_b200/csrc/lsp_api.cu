@@ -46,7 +46,7 @@ struct lsp_ctx {
   float *pmax = nullptr, *margin = nullptr;
   int *row_seq = nullptr, *row_pos = nullptr, *head_src = nullptr, *head_pos = nullptr;
   int32_t* prev_yhat = nullptr;  // [max_batch][max_len] argmax of the previous step per absolute position (-1 = none)
-  int* d_desc = nullptr;      // 7 arrays of (max_batch + 1) ints
+  int* d_desc = nullptr;      // 2 descriptors of 7 arrays of (max_batch + 1) ints
   int* d_scan = nullptr;      // 6 arrays of max_batch (run, commit, flags, tau, flips, flip base)
   float2* rope_cs = nullptr;
   unsigned* d_status = nullptr;
@@ -61,6 +61,12 @@ struct lsp_ctx {
   bool proposed = false;
   int score_rows = 0;
   int last_M = 0;
+  int lagged = 0;                   // lsp_generate keeps the block lengths on the device (see lsp_set_option key 4)
+  int lag_tail = 8;                 // ... until at most this many masked positions per sequence remain
+  // ring of result slots for the lagged loop: scan outputs + status word (pinned), completion and timing events
+  static constexpr int kRing = 4;
+  int* h_ring = nullptr;            // kRing x (6 max_batch + 4) ints
+  cudaEvent_t ring_done[kRing] = {}, ring_t0[kRing] = {}, ring_t1[kRing] = {};
   int kv_inplace = 0;               // K/V layout: 0 = staging planes + append copy, 1 = written in place (see lsp_set_option key 3)
   int last_attn_kernel = 0, last_attn_cluster = 1;   // what the last attention launch was (see lsp_get_counters)
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -136,16 +142,18 @@ void seg_collect(lsp_ctx* c) {
     if (e_ != cudaSuccess) return fail(c, LSP_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
   } while (0)
 
-StepDesc desc_of(const lsp_ctx* c) {
+// The device holds two descriptors (7 arrays of max_batch + 1 ints each); the synchronous path uses the first.
+StepDesc desc_of(const lsp_ctx* c, int which = 0) {
   const int s = c->max_batch + 1;
+  int* base = c->d_desc + (size_t)which * 7 * s;
   StepDesc d;
-  d.F = c->d_desc + 0 * s;
-  d.pend = c->d_desc + 1 * s;
-  d.N = c->d_desc + 2 * s;
-  d.row_off = c->d_desc + 3 * s;
-  d.head_off = c->d_desc + 4 * s;
-  d.Fp = c->d_desc + 5 * s;
-  d.Lc = c->d_desc + 6 * s;
+  d.F = base + 0 * s;
+  d.pend = base + 1 * s;
+  d.N = base + 2 * s;
+  d.row_off = base + 3 * s;
+  d.head_off = base + 4 * s;
+  d.Fp = base + 5 * s;
+  d.Lc = base + 6 * s;
   return d;
 }
 
@@ -188,7 +196,7 @@ Layout make_layout(const lsp_model_cfg* m, int max_batch, int max_len) {
   L.head_src = cv.take(R * 4);
   L.head_pos = cv.take(R * 4);
   L.prev_yhat = cv.take(R * 4);
-  L.desc = cv.take(7 * (size_t)(max_batch + 1) * 4);
+  L.desc = cv.take(2 * 7 * (size_t)(max_batch + 1) * 4);
   L.scan = cv.take(6 * (size_t)max_batch * 4);
   L.rope = cv.take((size_t)max_len * (m->head_dim / 2) * sizeof(float2));
   L.status = cv.take(256);
@@ -271,7 +279,7 @@ ScanParams scan_params(const lsp_ctx* c) {
 }
 
 // merge partials -> scores, scan, copy the scan outputs to the pinned mirror (async)
-int run_merge_scan(lsp_ctx* c, int rows, int n_tiles, const int* d_seq_off, int batch, bool count_flips) {
+int run_merge_scan(lsp_ctx* c, int rows, int n_tiles, const int* d_seq_off, int batch, bool count_flips, int* h_dst = nullptr) {
   if (rows > 0) {
     CU(launch_k(c->pdl, k_merge_partials, dim3((rows + 3) / 4), dim3(128), 0, c->stream, (const Top2*)c->part, n_tiles, rows, c->yhat,
                 c->pmax, c->margin));
@@ -287,6 +295,11 @@ int run_merge_scan(lsp_ctx* c, int rows, int n_tiles, const int* d_seq_off, int 
   launch_k(c->pdl, k_lsp_scan, dim3(batch), dim3(32), 0, c->stream, score, c->yhat, c->margin, d_seq_off, scan_params(c), o, o + mb,
                                           (uint32_t*)(o + 2 * mb), (float*)(o + 3 * mb));
   CU(cudaGetLastError());
+  if (h_dst) {        // a slot of the lagged loop's ring: scan outputs, then the status word
+    CU(cudaMemcpyAsync(h_dst, c->d_scan, 6 * (size_t)mb * 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaMemcpyAsync(h_dst + 6 * mb, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
+    return LSP_OK;
+  }
   CU(cudaMemcpyAsync(c->h_scan, c->d_scan, 6 * (size_t)mb * 4, cudaMemcpyDeviceToHost, c->stream));
   CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
   return LSP_OK;
@@ -309,9 +322,8 @@ int check_status(lsp_ctx* c) {
 // of the pass's own rows).  Reads the uploaded descriptor (F, row_off), Q from q, K/V from the cache and the staging
 // planes of layer l; writes out.  max_q: most query rows of one sequence; max_keys: most keys of one sequence.
 template <typename T>
-int run_attention(lsp_ctx* c, int l, const T* Qb, T* Att, int B, int maxQ, int max_keys, int inplace) {
+int run_attention(lsp_ctx* c, int l, const T* Qb, T* Att, const StepDesc& sd, int B, int maxQ, int max_keys, int inplace) {
   const lsp_model_cfg& m = c->m;
-  const StepDesc sd = desc_of(c);
   const int dh = m.head_dim, kvd = m.n_kv_heads * dh;
   const size_t plane = (size_t)c->max_rows * kvd;
   const size_t cplane = (size_t)c->max_batch * c->max_len * kvd;
@@ -377,37 +389,20 @@ int run_attention(lsp_ctx* c, int l, const T* Qb, T* Att, int B, int maxQ, int m
   return LSP_OK;
 }
 
+// Launch shape of one denoiser pass.  The row counts may be upper bounds of what the device-side descriptor says (the
+// lagged loop sizes a pass before it has read the previous block lengths): rows past the real ones are inert.
+struct PassDims {
+  int M = 0, Mh = 0;            // packed rows of the pass; rows that go through the LM head
+  int maxQ = 0, max_keys = 0;   // most rows / most keys of one sequence
+  double attn_bytes = 0, attn_flops = 0;      // algorithmic attention work per layer (accounting only)
+};
+
+// Enqueues one pass (Algorithm 1: forward pass, scores, scan) that reads descriptor sd on the device.
 template <typename T>
-int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
+int enqueue_pass(lsp_ctx* c, const StepDesc& sd, int B, const PassDims& pd, int* h_dst) {
   const lsp_model_cfg& m = c->m;
-  const int B = c->batch, s = c->max_batch + 1;
-  int* h = c->h_desc;
-  int M = 0, Mh = 0, maxQ = 0;
   const bool scattered = c->s.topology == 1;
-  for (int b = 0; b < B; ++b) {
-    const int pend = c->N[b] > 0 ? c->pend[b] : 0;
-    // rows past the pending block: the masked suffix (prefix topology) or the whole generation region (scattered)
-    const int tail = c->N[b] > 0 ? (scattered ? c->G[b] : c->N[b]) : 0;
-    const int rows = pend + tail;
-    h[0 * s + b] = c->F[b];
-    h[1 * s + b] = pend;
-    h[2 * s + b] = tail;
-    h[3 * s + b] = M;
-    h[4 * s + b] = Mh;
-    h[5 * s + b] = c->Fp[b];
-    M += rows;
-    Mh += c->N[b];
-    if (rows > maxQ) maxQ = rows;
-  }
-  h[3 * s + B] = M;
-  h[4 * s + B] = Mh;
-  if (M == 0) return fail(c, LSP_ERR_STATE, "lsp_denoise_step: every sequence is already fully committed");
-  const auto host_t0 = std::chrono::steady_clock::now();
-  CU(cudaEventRecord(c->ev0, c->stream));
-  // the step owns the first six arrays; the seventh (commit lengths) belongs to lsp_commit, whose upload from the same
-  // pinned mirror may still be in flight
-  CU(cudaMemcpyAsync(c->d_desc, h, 6 * (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
-  const StepDesc sd = desc_of(c);
+  const int M = pd.M, Mh = pd.Mh;
   const int d = m.d_model, dh = m.head_dim, qd = m.n_heads * dh, kvd = m.n_kv_heads * dh;
   T* X = (T*)c->X;
   T* Nrm = (T*)c->Nrm;
@@ -445,17 +440,9 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
       if (rc) return rc;
     }
     {
-      // algorithmic attention traffic: every key/value row of every sequence once per layer, plus Q and O
-      for (int b = 0; b < B; ++b) {
-        if (c->N[b] == 0) continue;
-        const double rows_b = c->pend[b] + (scattered ? c->G[b] : c->N[b]);
-        c->counters[CNT_ATTN_BYTES] += (2.0 * (c->F[b] + rows_b) * kvd + 2.0 * rows_b * qd) * sizeof(T);
-        c->counters[CNT_ATTN_FLOPS] += 4.0 * rows_b * (c->F[b] + rows_b) * qd;
-      }
-      int max_keys = 0;
-      for (int b = 0; b < B; ++b)
-        if (c->N[b] > 0) max_keys = std::max(max_keys, c->F[b] + c->pend[b] + (scattered ? c->G[b] : c->N[b]));
-      const int rc = run_attention<T>(c, l, Qb, Att, B, maxQ, max_keys, c->kv_inplace);
+      c->counters[CNT_ATTN_BYTES] += pd.attn_bytes;
+      c->counters[CNT_ATTN_FLOPS] += pd.attn_flops;
+      const int rc = run_attention<T>(c, l, Qb, Att, sd, B, pd.maxQ, pd.max_keys, c->kv_inplace);
       if (rc) return rc;
     }
     {
@@ -489,10 +476,60 @@ int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
   int rc = run_head<T>(c, Nrm, Mh, &n_tiles);
   if (rc) return rc;
   seg_begin(c, CLS_SCAN);
-  rc = run_merge_scan(c, Mh, n_tiles, sd.head_off, B, true);
+  rc = run_merge_scan(c, Mh, n_tiles, sd.head_off, B, true, h_dst);
   seg_end(c);
   count_launch(c, CLS_SCAN, 2);
   c->counters[CNT_STEPS] += 1;
+  return rc;
+}
+
+// Fills the pinned descriptor mirror from the host's state (arrays 0..5) and returns the pass's exact launch shape.
+PassDims host_descriptor(lsp_ctx* c) {
+  const lsp_model_cfg& m = c->m;
+  const int B = c->batch, s = c->max_batch + 1;
+  const bool scattered = c->s.topology == 1;
+  const double qd = (double)m.n_heads * m.head_dim, kvd = (double)m.n_kv_heads * m.head_dim;
+  int* h = c->h_desc;
+  PassDims pd;
+  for (int b = 0; b < B; ++b) {
+    const int pend = c->N[b] > 0 ? c->pend[b] : 0;
+    // rows past the pending block: the masked suffix (prefix topology) or the whole generation region (scattered)
+    const int tail = c->N[b] > 0 ? (scattered ? c->G[b] : c->N[b]) : 0;
+    const int rows = pend + tail;
+    h[0 * s + b] = c->F[b];
+    h[1 * s + b] = pend;
+    h[2 * s + b] = tail;
+    h[3 * s + b] = pd.M;
+    h[4 * s + b] = pd.Mh;
+    h[5 * s + b] = c->Fp[b];
+    pd.M += rows;
+    pd.Mh += c->N[b];
+    pd.maxQ = std::max(pd.maxQ, rows);
+    if (rows > 0) {
+      pd.max_keys = std::max(pd.max_keys, c->F[b] + rows);
+      // algorithmic attention traffic: every key/value row of the sequence once per layer, plus Q and O
+      pd.attn_bytes += (2.0 * (c->F[b] + rows) * kvd + 2.0 * rows * qd) * c->esz;
+      pd.attn_flops += 4.0 * rows * (c->F[b] + rows) * qd;
+    }
+  }
+  h[3 * s + B] = pd.M;
+  h[4 * s + B] = pd.Mh;
+  return pd;
+}
+
+template <typename T>
+int step_impl(lsp_ctx* c, lsp_step_rec* rec) {
+  const int B = c->batch, s = c->max_batch + 1;
+  const bool scattered = c->s.topology == 1;
+  const PassDims pd = host_descriptor(c);
+  const int M = pd.M, Mh = pd.Mh;
+  if (M == 0) return fail(c, LSP_ERR_STATE, "lsp_denoise_step: every sequence is already fully committed");
+  const auto host_t0 = std::chrono::steady_clock::now();
+  CU(cudaEventRecord(c->ev0, c->stream));
+  // the step owns the first six arrays; the seventh (commit lengths) belongs to lsp_commit, whose upload from the same
+  // pinned mirror may still be in flight
+  CU(cudaMemcpyAsync(c->d_desc, c->h_desc, 6 * (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
+  int rc = enqueue_pass<T>(c, desc_of(c), B, pd, nullptr);
   if (rc) return rc;
   CU(cudaEventRecord(c->ev1, c->stream));
   // host time spent queueing the pass (everything between the two event records)
@@ -642,6 +679,12 @@ int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sch
   cudaError_t e = cudaHostAlloc((void**)&c->h_desc, 7 * (size_t)(max_batch + 1) * 4, cudaHostAllocDefault);
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->h_scan, 6 * (size_t)max_batch * 4, cudaHostAllocDefault);
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->h_status, 16, cudaHostAllocDefault);
+  if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->h_ring, (size_t)lsp_ctx::kRing * (6 * max_batch + 4) * 4, cudaHostAllocDefault);
+  for (int i = 0; i < lsp_ctx::kRing && e == cudaSuccess; ++i) {
+    e = cudaEventCreateWithFlags(&c->ring_done[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreate(&c->ring_t0[i]);
+    if (e == cudaSuccess) e = cudaEventCreate(&c->ring_t1[i]);
+  }
   if (e == cudaSuccess) e = cudaEventCreate(&c->ev0);
   if (e == cudaSuccess) e = cudaEventCreate(&c->ev1);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->d_status, 0, 256, c->stream);
@@ -722,6 +765,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
     }
     c->kv_inplace = value ? 1 : 0;
   }
+  else if (key == 4) c->lagged = value ? 1 : 0;
   else return fail(c, LSP_ERR_ARG, "lsp_set_option: unknown key %d", key);
   return LSP_OK;
 }
@@ -729,6 +773,7 @@ int lsp_set_option(lsp_ctx* c, int key, int value) {
 int lsp_debug_set(lsp_ctx* c, int key, int value) {
   if (!c) return LSP_ERR_ARG;
   if (key == 28) c->attn_umma_min_rows = value;
+  else if (key == 31) c->lag_tail = value < 1 ? 1 : value;
   else if (key == 30) c->attn_cluster = value ? 1 : 0;
   else if (key == 3) c->async_ops = value;
   else if (key == 4) c->op_repeat = value < 1 ? 1 : value;
@@ -797,6 +842,180 @@ int lsp_denoise_step(lsp_ctx* c, lsp_step_rec* rec) {
   return c->m.dtype == 0 ? step_impl<float>(c, rec) : step_impl<bf16>(c, rec);
 }
 
+}  // extern "C"
+
+namespace {
+
+// Enqueues the commit kernel(s) of a step that read descriptor sd (whose Lc array holds the block lengths).
+// max_pend: the longest pending block (an upper bound is enough: it only sizes the copy's grid).
+int enqueue_commit(lsp_ctx* c, const StepDesc& sd, int B, int max_pend, int max_n) {
+  const lsp_model_cfg& m = c->m;
+  const size_t kvd = (size_t)m.n_kv_heads * m.head_dim;
+  const int row_v4 = (int)(kvd * c->esz / 16);
+  const size_t stage_plane_v4 = (size_t)c->max_rows * row_v4;
+  const size_t cache_seq_v4 = (size_t)c->max_len * row_v4;
+  const size_t cache_plane_v4 = (size_t)c->max_batch * cache_seq_v4;
+  size_t n_v4 = (size_t)max_pend * row_v4;
+  int chunks = (int)((n_v4 + 256 * 8 - 1) / (256 * 8));
+  if (chunks < 1) chunks = 1;
+  if (chunks > 64) chunks = 64;
+  dim3 grid(chunks, m.n_layers * 2, B);
+  seg_begin(c, CLS_COMMIT);
+  const bool scattered = c->s.topology == 1;
+  const bool copy = !c->kv_inplace;          // in-place layout: the pending block's K/V are already where they belong
+  if (!copy) grid = dim3(1, 1, B);
+  if ((!scattered || max_pend > 0) && (copy || !scattered)) {
+    launch_k(c->pdl, k_commit_append, dim3(grid), dim3(256), 0, c->stream, sd, (const uint4*)c->stage, (uint4*)c->kv_cache,
+                                                 stage_plane_v4, cache_plane_v4, cache_seq_v4, row_v4, c->yhat,
+                                                 c->tokens, c->tok_stride, scattered ? 0 : 1, copy ? 1 : 0);
+    count_launch(c, CLS_COMMIT);
+  }
+  if (scattered) {
+    // accept the L most confident masked positions wherever they are
+    const float* score = c->s.score == 1 ? c->margin : c->pmax;
+    launch_k(c->pdl, k_scatter_commit, dim3(B), dim3(256), (size_t)max_n * sizeof(float), c->stream, sd, score,
+             (const int32_t*)c->yhat, (const int*)c->head_pos, c->tokens, c->tok_stride);
+    count_launch(c, CLS_COMMIT);
+  }
+  seg_end(c);
+  CU(cudaGetLastError());
+  return LSP_OK;
+}
+
+// Algorithm 1's loop with the block lengths kept on the device (prefix topology).  Pass j+1 is enqueued before L_j has
+// been read back: the scan's L goes straight into the commit kernel, k_advance derives the next descriptor from it on
+// the device, and the host only needs the row counts to size the launches -- and those it knows one step late, because
+// a sequence's rows at step j+1 (pending block + masked suffix) are exactly its masked suffix at step j, N_j, which
+// follows from L_{j-1}.  The LM-head row count is an upper bound (N_j - 1); rows beyond the real ones are inert.
+// Near the end (at most lag_tail masked positions per sequence left) every step is read before the next one is sized,
+// so that no empty pass is launched after the last commit; a sequence that runs to its end earlier costs one empty pass.
+template <typename T>
+int generate_lagged(lsp_ctx* c, lsp_step_rec* recs, int max_recs, int* n_steps) {
+  const lsp_model_cfg& m = c->m;
+  const int B = c->batch, s = c->max_batch + 1, mb = c->max_batch, R = lsp_ctx::kRing;
+  const int slot_ints = 6 * mb + 4;
+  const double qd = (double)m.n_heads * m.head_dim, kvd = (double)m.n_kv_heads * m.head_dim;
+  std::vector<int> total(B);                       // prompt + generation length: F + rows of any pass of the sequence
+  for (int b = 0; b < B; ++b) total[b] = c->Fp[b] + c->N[b];
+  // host state = state before step `read` (results of steps < read have been applied)
+  int launched = 0, read = 0, used = 0, steps_done = 0;
+  int last_L = 1;                                  // longest block of the last step read (sizes the next append's grid)
+  auto apply_results = [&](int j) -> int {         // waits for step j, folds its block lengths into the host state
+    const int slot = j % R;
+    CU(cudaEventSynchronize(c->ring_done[slot]));
+    const int* r = c->h_ring + (size_t)slot * slot_ints;
+    if (r[6 * mb] != 0) {
+      memcpy(c->h_status, r + 6 * mb, 16);
+      return check_status(c);
+    }
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, c->ring_t0[slot], c->ring_t1[slot]);
+    c->timing_ms[6] += ms;
+    bool any = false;
+    for (int b = 0; b < B; ++b) any |= c->N[b] > 0;
+    for (int b = 0; b < B; ++b) {
+      const int L = c->N[b] > 0 ? r[mb + b] : 0;
+      if (any && recs && used < max_recs) {
+        lsp_step_rec& o = recs[used++];
+        o.step = c->step;
+        o.n_before = c->N[b];
+        o.rows = c->N[b] > 0 ? c->pend[b] + c->N[b] : 0;
+        o.l_run = r[b];
+        o.l_commit = r[mb + b];
+        o.flags = (unsigned)r[2 * mb + b];
+        memcpy(&o.tau_used, &r[3 * mb + b], 4);
+        o.ms = ms;
+        o.flips = c->N[b] > 0 ? r[4 * mb + b] : 0;
+        o.flip_base = c->N[b] > 0 ? r[5 * mb + b] : 0;
+      }
+      if (c->N[b] == 0) continue;
+      if (L < 1 || L > c->N[b]) return fail(c, LSP_ERR_STATE, "lagged loop: step %d proposed L[%d] = %d outside [1, %d]", j, b, L, c->N[b]);
+      if (!c->kv_inplace) c->counters[CNT_APPEND_BYTES] += 2.0 * c->pend[b] * kvd * c->esz * 2.0 * m.n_layers;
+      c->counters[CNT_TOKENS] += L;
+      c->F[b] += c->pend[b];
+      c->Fp[b] += L;
+      c->pend[b] = L;
+      c->N[b] -= L;
+    }
+    if (any) {
+      c->step += 1;
+      ++steps_done;
+      last_L = 1;
+      for (int b = 0; b < B; ++b) last_L = std::max(last_L, c->pend[b]);
+    }
+    return LSP_OK;
+  };
+  int rc = LSP_OK;
+  for (;;) {
+    // before sizing step `launched`, the host must know N of step launched - 1, i.e. have read step launched - 2
+    while (read < launched - 1) { rc = apply_results(read); if (rc) return rc; ++read; }
+    int remaining = 0, most = 0;
+    for (int b = 0; b < B; ++b) { remaining += c->N[b]; most = std::max(most, c->N[b]); }
+    // host state is now that before step launched - 1 (or before step 0).  Near the end, or when that step may have
+    // finished every sequence, read it too.
+    if (launched > read && (most <= c->lag_tail || remaining == 0)) { rc = apply_results(read); if (rc) return rc; ++read; }
+    remaining = 0;
+    for (int b = 0; b < B; ++b) remaining += c->N[b];
+    if (remaining == 0) break;
+    const bool exact = (read == launched);           // the host state is that of the step about to be launched
+    PassDims pd;
+    if (exact) {
+      pd = host_descriptor(c);
+      // the device descriptor of this step: the first one is uploaded; later ones were derived on the device (k_advance)
+      // from the same block lengths and are equal to the host's
+      if (launched == 0) CU(cudaMemcpyAsync(c->d_desc, c->h_desc, 6 * (size_t)s * 4, cudaMemcpyHostToDevice, c->stream));
+    } else {
+      // host state is that before step launched - 1: this step's rows of sequence b are N there (if it goes on at all)
+      for (int b = 0; b < B; ++b) {
+        const int rows = c->N[b] >= 2 ? c->N[b] : 0;
+        pd.M += rows;
+        pd.Mh += rows > 0 ? rows - 1 : 0;
+        pd.maxQ = std::max(pd.maxQ, rows);
+        if (rows > 0) {
+          pd.max_keys = std::max(pd.max_keys, total[b]);
+          pd.attn_bytes += (2.0 * total[b] * kvd + 2.0 * rows * qd) * c->esz;
+          pd.attn_flops += 4.0 * rows * (double)total[b] * qd;
+        }
+      }
+      if (pd.M == 0) {            // every unfinished sequence has one masked position left: the step in flight ends them
+        rc = apply_results(read); if (rc) return rc; ++read;
+        continue;
+      }
+    }
+    const int par = launched & 1, slot = launched % R;
+    const StepDesc sd = desc_of(c, par);
+    CU(cudaEventRecord(c->ring_t0[slot], c->stream));
+    rc = enqueue_pass<T>(c, sd, B, pd, c->h_ring + (size_t)slot * slot_ints);
+    if (rc) return rc;
+    CU(cudaEventRecord(c->ring_t1[slot], c->stream));
+    CU(cudaEventRecord(c->ring_done[slot], c->stream));
+    // commit with the scan's own block lengths, then the next step's descriptor
+    StepDesc sc = sd;
+    sc.Lc = c->d_scan + mb;
+    int max_pend = 0;
+    if (exact) { for (int b = 0; b < B; ++b) if (c->N[b] > 0) max_pend = std::max(max_pend, c->pend[b]); }
+    else max_pend = std::min(pd.maxQ, std::max(8, 2 * last_L));
+    rc = enqueue_commit(c, sc, B, max_pend, 0);
+    if (rc) return rc;
+    launch_k(c->pdl, k_advance, dim3(1), dim3(32), 0, c->stream, sd, c->d_desc + (size_t)(par ^ 1) * 7 * s, s,
+             (const int32_t*)(c->d_scan + mb), B);
+    CU(cudaGetLastError());
+    count_launch(c, CLS_COMMIT);
+    c->last_M = pd.M;
+    c->score_rows = pd.Mh;
+    ++launched;
+  }
+  while (read < launched) { rc = apply_results(read); if (rc) return rc; ++read; }
+  CU(cudaStreamSynchronize(c->stream));
+  c->proposed = false;
+  if (n_steps) *n_steps = steps_done;
+  return LSP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
 int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
   if (!c) return LSP_ERR_ARG;
   if (!c->proposed) return fail(c, LSP_ERR_STATE, "lsp_commit without a preceding lsp_denoise_step");
@@ -815,38 +1034,13 @@ int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
   CU(cudaMemcpyAsync(c->d_desc + 6 * s, hl, (size_t)B * 4, cudaMemcpyHostToDevice, c->stream));
   const lsp_model_cfg& m = c->m;
   const size_t kvd = (size_t)m.n_kv_heads * m.head_dim;
-  const int row_v4 = (int)(kvd * c->esz / 16);
-  const size_t stage_plane_v4 = (size_t)c->max_rows * row_v4;
-  const size_t cache_seq_v4 = (size_t)c->max_len * row_v4;
-  const size_t cache_plane_v4 = (size_t)c->max_batch * cache_seq_v4;
-  size_t n_v4 = (size_t)max_pend * row_v4;
-  int chunks = (int)((n_v4 + 256 * 8 - 1) / (256 * 8));
-  if (chunks < 1) chunks = 1;
-  if (chunks > 64) chunks = 64;
-  dim3 grid(chunks, m.n_layers * 2, B);
-  seg_begin(c, CLS_COMMIT);
   const bool scattered = c->s.topology == 1;
-  const bool copy = !c->kv_inplace;          // in-place layout: the pending block's K/V are already where they belong
-  if (!copy) grid = dim3(1, 1, B);
-  if ((!scattered || max_pend > 0) && (copy || !scattered)) {
-    launch_k(c->pdl, k_commit_append, dim3(grid), dim3(256), 0, c->stream, desc_of(c), (const uint4*)c->stage, (uint4*)c->kv_cache,
-                                                 stage_plane_v4, cache_plane_v4, cache_seq_v4, row_v4, c->yhat,
-                                                 c->tokens, c->tok_stride, scattered ? 0 : 1, copy ? 1 : 0);
-    count_launch(c, CLS_COMMIT);
-  }
-  if (scattered) {
-    // accept the L most confident masked positions wherever they are
-    int max_n = 0;
-    for (int b = 0; b < B; ++b) if (c->N[b] > max_n) max_n = c->N[b];
-    const float* score = c->s.score == 1 ? c->margin : c->pmax;
-    launch_k(c->pdl, k_scatter_commit, dim3(B), dim3(256), (size_t)max_n * sizeof(float), c->stream, desc_of(c), score,
-             (const int32_t*)c->yhat, (const int*)c->head_pos, c->tokens, c->tok_stride);
-    count_launch(c, CLS_COMMIT);
-  }
-  seg_end(c);
+  int max_n = 0;
+  for (int b = 0; b < B; ++b) if (c->N[b] > max_n) max_n = c->N[b];
+  const int rc = enqueue_commit(c, desc_of(c), B, max_pend, max_n);
+  if (rc) return rc;
   for (int b = 0; b < B; ++b)
-    if (c->N[b] > 0 && copy) c->counters[CNT_APPEND_BYTES] += 2.0 * c->pend[b] * kvd * c->esz * 2.0 * m.n_layers;
-  CU(cudaGetLastError());
+    if (c->N[b] > 0 && !c->kv_inplace) c->counters[CNT_APPEND_BYTES] += 2.0 * c->pend[b] * kvd * c->esz * 2.0 * m.n_layers;
   for (int b = 0; b < B; ++b) {
     if (c->N[b] == 0) continue;
     c->F[b] += c->pend[b];
@@ -863,6 +1057,8 @@ int lsp_commit(lsp_ctx* c, const int32_t* L_override) {
 int lsp_generate(lsp_ctx* c, lsp_step_rec* recs, int max_recs, int* n_steps) {
   if (!c) return LSP_ERR_ARG;
   if (!c->tokens) return fail(c, LSP_ERR_STATE, "lsp_generate before lsp_begin");
+  if (c->lagged && c->s.topology == 0 && !c->timing && !c->proposed)
+    return c->m.dtype == 0 ? generate_lagged<float>(c, recs, max_recs, n_steps) : generate_lagged<bf16>(c, recs, max_recs, n_steps);
   int steps = 0, used = 0;
   std::vector<lsp_step_rec> tmp(c->batch);
   for (;;) {
@@ -1007,8 +1203,8 @@ int lsp_op_attention(lsp_ctx* c, int layer, const void* q, const void* k_new, co
   char* stK = c->stage + (size_t)(2 * layer) * plane;
   CU(cudaMemcpyAsync(stK, k_new, (size_t)M * kvd * c->esz, cudaMemcpyDeviceToDevice, c->stream));
   CU(cudaMemcpyAsync(stK + plane, v_new, (size_t)M * kvd * c->esz, cudaMemcpyDeviceToDevice, c->stream));
-  const int rc = c->m.dtype == 0 ? run_attention<float>(c, layer, (const float*)q, (float*)out, batch, maxQ, max_keys, 0)
-                                 : run_attention<bf16>(c, layer, (const bf16*)q, (bf16*)out, batch, maxQ, max_keys, 0);
+  const int rc = c->m.dtype == 0 ? run_attention<float>(c, layer, (const float*)q, (float*)out, desc_of(c), batch, maxQ, max_keys, 0)
+                                 : run_attention<bf16>(c, layer, (const bf16*)q, (bf16*)out, desc_of(c), batch, maxQ, max_keys, 0);
   if (rc) return rc;
   CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
   CU(cudaStreamSynchronize(c->stream));
@@ -1174,6 +1370,12 @@ int lsp_destroy(lsp_ctx* c) {
   if (c->h_desc) cudaFreeHost(c->h_desc);
   if (c->h_scan) cudaFreeHost(c->h_scan);
   if (c->h_status) cudaFreeHost(c->h_status);
+  if (c->h_ring) cudaFreeHost(c->h_ring);
+  for (int i = 0; i < lsp_ctx::kRing; ++i) {
+    if (c->ring_done[i]) cudaEventDestroy(c->ring_done[i]);
+    if (c->ring_t0[i]) cudaEventDestroy(c->ring_t0[i]);
+    if (c->ring_t1[i]) cudaEventDestroy(c->ring_t1[i]);
+  }
   if (c->ev0) cudaEventDestroy(c->ev0);
   if (c->ev1) cudaEventDestroy(c->ev1);
   for (cudaEvent_t e : c->seg_ev) cudaEventDestroy(e);

@@ -42,6 +42,9 @@ extern "C" {
  * tcgen05 attention:
  *   28 fewest (query row x group head) rows of a (sequence, KV head) for which the tcgen05 kernel is used (default 0)
  *   30 it splits a row tile's keys over a thread block cluster when there are few CTAs (1, default)
+ * decode loop:
+ *   31 with device-resident block lengths (lsp_set_option key 4), lsp_generate reads every step before sizing the next
+ *      once at most this many masked positions per sequence remain (default 8)
  * Unknown key: LSP_ERR_ARG. */
 int lsp_debug_set(lsp_ctx* ctx, int key, int value);
 

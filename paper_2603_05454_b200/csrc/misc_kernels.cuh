@@ -16,6 +16,15 @@ __global__ void k_assemble_embed(StepDesc sd, int batch, const int32_t* __restri
                                  int* __restrict__ head_src, int* __restrict__ head_pos, int scattered) {
   pdl_begin();
   const int r = blockIdx.x;
+  // The grid may be larger than the pass (a host that sizes launches from an upper bound of the row counts): rows past
+  // the last real one are zero vectors that belong to no sequence, and the spare head slots point at row 0.
+  if (r >= sd.head_off[batch] && threadIdx.x == 0) head_src[r] = 0;
+  if (r >= sd.row_off[batch]) {
+    if (threadIdx.x == 0) { row_seq[r] = -1; row_pos[r] = 0; }
+    uint4* z = reinterpret_cast<uint4*>(X + (size_t)r * d);
+    for (int i = threadIdx.x; i < d * (int)sizeof(T) / 16; i += blockDim.x) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
   int b = 0;
   while (b + 1 < batch && r >= sd.row_off[b + 1]) ++b;
   const int j = r - sd.row_off[b];
@@ -300,6 +309,34 @@ __global__ void k_commit_append(StepDesc sd, const uint4* __restrict__ stage, ui
     int32_t* t = tokens + (size_t)b * tok_stride + sd.Fp[b];
     for (int i = threadIdx.x; i < L; i += blockDim.x) t[i] = yhat[ho + i];
   }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Next step's descriptor, computed on the device from this step's and the scan's block lengths (prefix topology), so
+// that the host can enqueue the next pass without reading L back first:
+//   F += pend;  pend = L;  N -= L;  Fp += L;  rows = pend + N (0 once N = 0);  row_off / head_off = prefix sums.
+// One thread; runs after the commit kernel of the step (which still reads the current descriptor).
+// ---------------------------------------------------------------------------------------------
+__global__ void k_advance(StepDesc cur, int* __restrict__ nxt, int stride, const int32_t* __restrict__ L_commit, int batch) {
+  pdl_begin();
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  int M = 0, Mh = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int N = cur.N[b];
+    const int L = N > 0 ? L_commit[b] : 0;
+    const int pend = N > 0 ? cur.pend[b] : 0;
+    const int N2 = N - L;
+    nxt[0 * stride + b] = cur.F[b] + pend;
+    nxt[1 * stride + b] = N2 > 0 ? L : 0;
+    nxt[2 * stride + b] = N2;
+    nxt[3 * stride + b] = M;
+    nxt[4 * stride + b] = Mh;
+    nxt[5 * stride + b] = cur.Fp[b] + L;
+    M += N2 > 0 ? L + N2 : 0;
+    Mh += N2;
+  }
+  nxt[3 * stride + batch] = M;
+  nxt[4 * stride + batch] = Mh;
 }
 
 // ---------------------------------------------------------------------------------------------
