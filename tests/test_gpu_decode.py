@@ -35,7 +35,7 @@ def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, 
     decode(om, prompt[0].numpy(), G, make_is_delim(*delim), oracle_policy(sched), max_steps=1,
            on_step=lambda rec, lg, k, v: zr.append(float(np.sqrt((lg * lg).mean()))))
     tol_z = tol_logit(shape.dtype, zr[0], shape.n_layers)
-    tol_p = tol_prob(shape.dtype, tol_z)
+    tol_p = tol_prob(shape.dtype, zr[0], shape.n_layers)
     sched.flag_tol = tol_z if sched.score == 1 else tol
     sched.tie_tol = tol_z
     otok, orecs, (ock, ocv) = decode(om, prompt[0].numpy(), G, make_is_delim(*delim), oracle_policy(sched),
