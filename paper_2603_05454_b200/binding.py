@@ -62,6 +62,7 @@ def _load():
     l.lsp_set_sched.argtypes = [C.c_void_p, C.POINTER(SchedCfgC)]
     l.lsp_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int]
     l.lsp_debug_set.argtypes = [C.c_void_p, C.c_int, C.c_int]      # internal (csrc/lsp_tuning.h), not in EXPORTS
+    l.lsp_debug_wait_selftest.argtypes = [C.c_void_p, C.c_int]
     l.lsp_begin.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int]
     l.lsp_denoise_step.argtypes = [C.c_void_p, C.POINTER(StepRec)]
     l.lsp_commit.argtypes = [C.c_void_p, C.c_void_p]
@@ -198,6 +199,10 @@ class LSPDecoder:
     def debug_set(self, key: int, value: int):
         """Internal tuning and benchmark knobs (csrc/lsp_tuning.h); not part of the public interface."""
         self._check(lib.lsp_debug_set(self._h, key, value))
+
+    def wait_selftest(self, limit_us: int = 200):
+        """Internal (csrc/lsp_tuning.h): lets a bounded device-side wait run out; raises LSPError(-6)."""
+        self._check(lib.lsp_debug_wait_selftest(self._h, limit_us))
 
     # -- Algorithm 1
     def begin(self, tokens: torch.Tensor, prompt_len, gen_len):

@@ -55,8 +55,9 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-// Bounded wait.  Returns false after UM_WAIT_NS or when another role has raised the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+// Bounded wait.  Returns false after limit_ns (default UM_WAIT_NS) or when another role has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint64_t limit_ns = UM_WAIT_NS) {
   uint64_t t0 = 0;
   for (uint32_t spin = 0;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -64,7 +65,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const uint64_t now = globaltimer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > UM_WAIT_NS) return false;
+      else if (now - t0 > limit_ns) return false;
+    }
+  }
+}
+
+// Self-test of the bounded-wait protocol: one thread waits on a barrier that nobody ever arrives at, gives up after
+// limit_ns and reports it exactly as the kernels' roles do: (code 1, site 99) in the status word.  Nothing else runs,
+// nothing is in flight, the context stays usable.
+__global__ void k_wait_selftest(unsigned* status, unsigned long long limit_ns) {
+  __shared__ uint64_t never;
+  __shared__ uint32_t no_abort;
+  if (threadIdx.x == 0) {
+    no_abort = 0;
+    mbar_init(smem_u32(&never), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!mbar_wait(smem_u32(&never), 0u, &no_abort, (uint64_t)limit_ns)) {
+      atomicExch(status, 1u);
+      status[1] = 99u;
     }
   }
 }

@@ -1211,6 +1211,20 @@ int lsp_op_attention(lsp_ctx* c, int layer, const void* q, const void* k_new, co
   return check_status(c);
 }
 
+int lsp_debug_wait_selftest(lsp_ctx* c, int limit_us) {
+  if (!c) return LSP_ERR_ARG;
+#ifndef LSP_NO_UMMA
+  if (limit_us < 1 || limit_us > 1000000) return fail(c, LSP_ERR_ARG, "lsp_debug_wait_selftest: limit outside [1 us, 1 s]");
+  k_wait_selftest<<<1, 32, 0, c->stream>>>(c->d_status, (unsigned long long)limit_us * 1000ull);
+  CU(cudaGetLastError());
+  CU(cudaMemcpyAsync(c->h_status, c->d_status, 16, cudaMemcpyDeviceToHost, c->stream));
+  CU(cudaStreamSynchronize(c->stream));
+  return check_status(c);
+#else
+  return fail(c, LSP_ERR_SHAPE, "built without the tcgen05 kernels");
+#endif
+}
+
 int lsp_last_timing(lsp_ctx* c, float* ms) {
   if (!c || !ms) return LSP_ERR_ARG;
   CU(cudaStreamSynchronize(c->stream));

@@ -48,6 +48,12 @@ extern "C" {
  * Unknown key: LSP_ERR_ARG. */
 int lsp_debug_set(lsp_ctx* ctx, int key, int value);
 
+/* Exercises the bounded-wait recovery path without touching any data: launches one thread that waits, for limit_us
+ * microseconds, on a barrier nothing arrives at, and then records the expiry in the context's status word the way the
+ * GEMM and attention kernels do.  Returns what a step would return in that situation: LSP_ERR_DEVICE_TIMEOUT (site 99
+ * in lsp_last_error), with the status word and the split-K counters cleared again, so that the next call runs normally. */
+int lsp_debug_wait_selftest(lsp_ctx* ctx, int limit_us);
+
 #ifdef __cplusplus
 }
 #endif

@@ -2,6 +2,8 @@
 
   gemm   one linear layer  out = A W^T  (or the residual / SwiGLU epilogues) at a given M, N, K; the weights are
          read from a ring of copies larger than the L2 cache so that every launch streams them from HBM
+  layer  the four GEMMs of one transformer layer (fused QKV, O, gate/up + SwiGLU, down) of a model shape given by
+         --d --heads --kv-heads --ffn (default: a shape the tile heuristics were not fitted on: 5120, 40/8, 13824)
   head   the fused LM head + confidence reduction + scan on M hidden rows
   decode per-class kernel times of a full decode of a named workload (same figures bench.py reports)
 
@@ -157,11 +159,14 @@ def bench_decode(name, decodes=1, layers=0, max_passes=0, fast_init=False, opts=
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("what", choices=["gemm", "head", "decode"])
+    ap.add_argument("what", choices=["gemm", "layer", "head", "decode"])
     ap.add_argument("--M", type=int, nargs="+", default=[128])
     ap.add_argument("--N", type=int, default=4096)
     ap.add_argument("--K", type=int, default=4096)
     ap.add_argument("--V", type=int, default=126464)
+    ap.add_argument("--heads", type=int, default=40)
+    ap.add_argument("--kv-heads", type=int, default=8)
+    ap.add_argument("--ffn", type=int, default=13824)
     ap.add_argument("--d", type=int, default=4096)
     ap.add_argument("--op", type=int, default=0)
     ap.add_argument("--reps", type=int, default=50)
@@ -178,6 +183,13 @@ def main():
     if a.what == "gemm":
         for m in a.M:
             print(json.dumps(bench_gemm(m, a.N, a.K, a.op, a.reps, a.copies, opts=a.opt)), flush=True)
+    elif a.what == "layer":
+        d = a.d if a.d != 4096 else 5120
+        qd, kvd = a.heads * 128, a.kv_heads * 128
+        for m in a.M:
+            for name, (n, k, op) in (("qkv", (qd + 2 * kvd, d, 0)), ("o", (d, qd, 1)), ("gate_up", (a.ffn, d, 2)),
+                                     ("down", (d, a.ffn, 1))):
+                print(json.dumps(dict(gemm=name, **bench_gemm(m, n, k, op, a.reps, a.copies, opts=a.opt))), flush=True)
     elif a.what == "head":
         for m in a.M:
             print(json.dumps(bench_head(m, a.V, a.d, a.reps)), flush=True)

@@ -178,3 +178,50 @@ def test_linear_bf16_seeded_random_shapes_and_kernel_options():
         np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05, err_msg=tag)
         done += 1
     dec.close()
+
+
+def test_bounded_wait_expiry_is_reported_and_the_context_stays_usable():
+    """A device-side wait that runs out (a barrier nothing arrives at, 200 microseconds) comes back as
+    LSP_ERR_DEVICE_TIMEOUT with the site in the message; the status word is cleared, and the next GEMM is correct."""
+    from paper_2603_05454_b200 import LSPError
+    dec = _dec("bf16")
+    A = S.normal((70, 192), 3, 1, 1.0, torch.bfloat16, DEV)
+    W = S.normal((144, 192), 3, 2, 0.05, torch.bfloat16, DEV)
+    out = torch.empty(70, 144, dtype=torch.bfloat16, device=DEV)
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    ref = dlm.round_bf16(f64(A) @ f64(W).T)
+    for _ in range(2):
+        with pytest.raises(LSPError) as e:
+            dec.wait_selftest(200)
+        assert e.value.code == -6 and "site 99" in str(e.value)
+        dec.op_linear(0, A, W, None, out)               # synchronises and checks the status word: must be clean again
+        np.testing.assert_allclose(f64(out), ref, rtol=1.0 / 128, atol=np.abs(ref).max() / 128 * 0.05)
+    dec.close()
+
+
+@pytest.mark.parametrize("M", [1, 48, 128, 200, 256, 384, 640, 1500])
+def test_linear_bf16_third_model_shape(M):
+    """A model shape none of the tile heuristics were fitted on (d 5120, 40/8 heads of 128, FFN 13824): the fused QKV
+    width 7168, the O and down projections, the SwiGLU pair GEMM, at row counts of every regime."""
+    dec = _dec("bf16")
+    d, qd, kvd, f = 5120, 40 * 128, 8 * 128, 13824
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    rtol = 1.0 / 128
+    for (N, K, op) in ((qd + 2 * kvd, d, 0), (d, qd, 1), (f, d, 2), (d, f, 1)):
+        A = S.normal((M, K), 5, 1, 1.0, torch.bfloat16, DEV)
+        W = S.normal((N, K), 5, 2, 0.03, torch.bfloat16, DEV)
+        W2 = S.normal((N, K), 5, 3, 0.03, torch.bfloat16, DEV) if op == 2 else None
+        out = S.normal((M, N), 5, 4, 1.0, torch.bfloat16, DEV)
+        x0 = f64(out)
+        dec.op_linear(op, A, W, W2, out)
+        a, w = f64(A), f64(W)
+        if op == 0:
+            ref = a @ w.T
+        elif op == 1:
+            ref = x0 + a @ w.T
+        else:
+            g, u = a @ w.T, a @ f64(W2).T
+            ref = g / (1 + np.exp(-g)) * u
+        np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * (2 if op == 2 else 1),
+                                   atol=rtol * np.abs(ref).max() * 0.05, err_msg=f"M={M} N={N} K={K} op={op}")
+    dec.close()
