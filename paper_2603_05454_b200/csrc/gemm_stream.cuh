@@ -1,7 +1,7 @@
 // Persistent bf16 GEMM on tcgen05, built for the weight-streaming regime (at most 256 activation rows: the shrinking
 // suffix of late decode steps) and also used, with whole tiles per CTA, for larger problems.
 //
-//   acc[m, c] = sum_k A[m, k] * Wt[c, k]        same operands, tiles and fused epilogues as gemm_umma.cuh
+//   acc[m, c] = sum_k A[m, k] * Wt[c, k]        operands, descriptors and fused epilogues: gemm_umma.cuh
 //
 // With M <= 256 a layer GEMM is bound by reading its weights from HBM once (at the upper end the tensor cores need
 // about as long), so the kernel is built around one uninterrupted stream of weight tiles per SM, each weight tile
@@ -787,7 +787,6 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
 // for the accumulators, scratch or counters too small for a split grid, too little shared memory).
 template <typename Epi>
 int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn) {
-  if (!st.use_stream) return 0;
   const int per_tile = Epi::kDual ? bn / 2 : bn;
   const long n_tiles = (NP + per_tile - 1) / per_tile;
   int mt;
@@ -796,9 +795,9 @@ int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn) {
     // layer GEMMs: two row tiles per CTA (each weight tile is used for all rows while it is in shared memory); the LM
     // head has hundreds of column tiles, so two row groups of whole 128 x 256 tiles keep double-buffered accumulators
     // and run 1.5 x faster there (the second row group finds its weight tile in L2)
-    mt = (Epi::kReduce && st.stream_two_tiles) ? 1 : (st.stream_two_tiles == 1 ? 2 : (st.stream_two_tiles == 2 ? 1 : 0));
+    mt = (Epi::kReduce || st.stream_two_tiles == 2) ? 1 : 2;
   }
-  else if (st.stream_big_mt != 3) mt = st.stream_big_mt;   // 0 = leave large problems to the tiled kernel
+  else if (st.stream_big_mt == 1 || st.stream_big_mt == 2) mt = st.stream_big_mt;
   else {
     // 256 x 256 tiles (two row tiles per CTA) need a third less operand data per flop than 128 x 256 ones, which the
     // SM's shared-memory fill rate cannot quite sustain: they measure about 1.25 x faster when both fill the SMs equally

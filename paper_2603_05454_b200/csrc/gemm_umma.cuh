@@ -1,19 +1,16 @@
-// bf16 GEMM on the 5th-generation tensor cores (tcgen05) for sm_100a.
+// bf16 GEMM on the 5th-generation tensor cores (tcgen05) for sm_100a: the parts shared by every kernel that uses them.
 //
 //   acc[m, c] = sum_k A[m, k] * Wt[c, k]        A: [M, K] bf16 row-major, Wt: weight rows, K-major, fp32 accumulate
 //
-// One CTA computes a 128 x BN accumulator tile that lives in tensor memory (TMEM).  Operand tiles are brought
-// into 128-byte-swizzled shared memory by TMA (cp.async.bulk.tensor, no multicast) through a ring of stages
-// guarded by mbarriers; a single thread issues tcgen05.mma (M = 128, N = BN, K = 16 per instruction) and
-// releases each stage with tcgen05.commit; four epilogue warps read the accumulators back with tcgen05.ld
-// (each thread owns one output row) and run the fused epilogue (store / residual / SwiGLU / rotary+KV staging /
-// LM-head top-2 + log-sum-exp reduction).
+// This header holds the PTX wrappers (mbarrier with bounded waits, TMA tile loads without multicast, tcgen05.mma /
+// .commit / .ld), the shared-memory and instruction descriptors, the vectorised fused epilogues (store / residual /
+// SwiGLU / rotary + K/V staging), the host state (tensor-map cache, tuning fields) and the dispatch that picks tile
+// width and row tiles per CTA.  The kernel itself is the persistent k_gemm_stream of gemm_stream.cuh; the attention
+// kernel (attention_umma.cuh) uses the same wrappers.
 //
 // The B tile is two TMA boxes of BN/2 weight rows each (possibly from two tensors), so accumulator columns
 // c and c + BN/2 of one thread hold the pair an element-wise fusion needs (gate/up, rotate-half partners).
-//
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = epilogue.
-// Every wait is bounded by wall-clock time; on expiry the kernel records (code, site) in a status word, lets
+// Every wait is bounded by wall-clock time; on expiry a kernel records (code, site) in a status word, lets
 // all roles drain and returns, so a protocol error can never hang the device.
 #pragma once
 #include <cuda.h>
@@ -28,7 +25,6 @@ namespace lsp {
 
 constexpr int UM_BM = 128;
 constexpr int UM_BK = 64;                 // bf16 elements = one 128-byte swizzle row
-constexpr int UM_THREADS = 192;
 constexpr int UM_MAX_STAGES = 12;
 constexpr uint64_t UM_WAIT_NS = 2000000000ull;   // 2 s
 
@@ -237,271 +233,6 @@ __device__ __forceinline__ void epi16(const EpiQKVRope<bf16>& e, int m, int j, c
   p1[1] = pack8(r1 + 8);
 }
 
-// ---- the kernel -------------------------------------------------------------------------------------------
-struct UmmaArgs {
-  int M;        // activation rows
-  int n_pairs;  // dual: pair indices (each tile covers BN/2); plain: output columns (each tile covers BN)
-  int K;
-  int num_kb;   // K / 64
-  int stages;
-  int a_rows;   // rows of the activation box (8..128): a single-tile launch loads only the rows that exist (rounded up);
-                // accumulator rows beyond them are computed from whatever the stage holds and are never stored
-  int m_fast;   // 1: blockIdx.x walks the row tiles (keeps one weight tile hot in L2 across the rows), 0: the column tiles
-  int splits;        // split-K factor (blockIdx.z); 1 = none
-  int kb_per_split;  // k-blocks per split (the last split may get fewer)
-  float* scratch;    // split-K partial tiles: [tile][split][128][BN] fp32
-  unsigned* counters;// split-K arrival counters, one per output tile, zero between launches
-  unsigned* status;
-};
-
-template <int BN>
-constexpr int umma_stage_bytes() { return UM_BM * UM_BK * 2 + BN * UM_BK * 2; }   // with a full activation tile
-
-// Split-K epilogue: publishes this CTA's partial tile; the CTA that arrives last at the tile sums all partials in
-// split order (deterministic) and runs the fused epilogue.  Returns false when the launch is not split.
-template <int BN, typename Epi>
-__device__ __forceinline__ bool splitk_epilogue(const UmmaArgs& args, const Epi& epi, uint32_t tmem_base, int q, int lane,
-                                                int m, int m0, int tile, volatile uint32_t* epi_last) {
-  if constexpr (Epi::kReduce) {
-    return false;
-  } else {
-    if (args.splits <= 1) return false;
-    constexpr int HALF = BN / 2;
-
-      tc_fence_after();
-      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
-      const int n_col_tiles = args.m_fast ? gridDim.y : gridDim.x;
-      const int tile_lin = (m0 / UM_BM) * n_col_tiles + tile;
-      const int r_in = q * 32 + lane;
-      float* base = args.scratch + (size_t)tile_lin * args.splits * (UM_BM * BN);
-      float* mine = base + ((size_t)blockIdx.z * UM_BM + r_in) * BN;
-#pragma unroll 1
-      for (int c = 0; c < BN; c += 16) {
-        float v[16];
-        tc_ld16(t_row + c, v);
-        if (m < args.M) {
-          float4* d4 = reinterpret_cast<float4*>(mine + c);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-        }
-      }
-      __threadfence();
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (threadIdx.x == 64) {
-        const unsigned old = atomicAdd(args.counters + tile_lin, 1u);
-        if (old == (unsigned)args.splits - 1u) {
-          args.counters[tile_lin] = 0;        // ready for the next launch
-          *epi_last = 1;
-        }
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (*epi_last) {
-        __threadfence();
-        const float* row = base + (size_t)r_in * BN;
-        constexpr int CH = Epi::kDual ? HALF : BN;
-        const int j0 = tile * CH;
-#pragma unroll 1
-        for (int c = 0; c < CH; c += 16) {
-          float a0[16], a1[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
-          if (m < args.M && j0 + c < args.n_pairs) {
-            for (int sp = 0; sp < args.splits; ++sp) {
-              const float4* p0 = reinterpret_cast<const float4*>(row + (size_t)sp * UM_BM * BN + c);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const float4 t = __ldcg(p0 + i);
-                a0[4 * i] += t.x; a0[4 * i + 1] += t.y; a0[4 * i + 2] += t.z; a0[4 * i + 3] += t.w;
-              }
-              if (Epi::kDual) {
-                const float4* p1 = reinterpret_cast<const float4*>(row + (size_t)sp * UM_BM * BN + HALF + c);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const float4 t = __ldcg(p1 + i);
-                  a1[4 * i] += t.x; a1[4 * i + 1] += t.y; a1[4 * i + 2] += t.z; a1[4 * i + 3] += t.w;
-                }
-              }
-            }
-            epi16(epi, m, j0 + c, a0, a1);
-          }
-        }
-      }
-    return true;
-  }
-}
-
-template <int BN, typename Epi>
-__global__ void __launch_bounds__(UM_THREADS, 1)
-k_gemm_umma(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
-            const __grid_constant__ CUtensorMap map_b1, UmmaArgs args, Epi epi) {
-  extern __shared__ uint8_t smem_raw[];
-  pdl_release();
-  constexpr int B_HALF_BYTES = (BN / 2) * UM_BK * 2;
-  constexpr int HALF = BN / 2;
-  const int A_BYTES = args.a_rows * UM_BK * 2;             // a multiple of 1024: the weight tile stays swizzle-aligned
-  const int STAGE_BYTES = A_BYTES + 2 * B_HALF_BYTES;
-  // 1024-byte alignment for the swizzled tiles
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  const int S = args.stages;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * STAGE_BYTES);
-  // bars[0..S) = full, bars[S..2S) = empty, bars[2S] = accumulator ready
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * S + 1);
-  volatile uint32_t* abort_flag = tmem_slot + 1;
-  volatile uint32_t* epi_fail = tmem_slot + 2;     // set when any epilogue warp's wait expired
-  volatile uint32_t* epi_last = tmem_slot + 3;     // split-K: this CTA arrived last at its tile
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = (args.m_fast ? blockIdx.x : blockIdx.y) * UM_BM;
-  const int tile = args.m_fast ? blockIdx.y : blockIdx.x;
-  // weight rows of the two boxes
-  int row_b0, row_b1;
-  if (Epi::kDual) {
-    row_b0 = epi.row0(tile * HALF);
-    row_b1 = epi.row1(tile * HALF);
-  } else {
-    row_b0 = tile * BN;
-    row_b1 = tile * BN + HALF;
-  }
-  const uint32_t bar_base = smem_u32(bars);
-  auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
-  const uint32_t acc_bar = bar_base + 8u * (2 * S);
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
-    }
-    mbar_init(acc_bar, 1);
-    *abort_flag = 0;
-    *epi_fail = 0;
-    *epi_last = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"((uint32_t)BN)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();          // barriers and tensor memory are set up; from here on the kernel reads what its predecessor wrote
-  const int kb0 = blockIdx.z * args.kb_per_split;
-  const int num_kb = min(args.kb_per_split, args.num_kb - kb0);
-
-  if (warp == 0) {
-    // ---------------- TMA producer ----------------
-    if (lane == 0) {
-      int issued = 0;
-      bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % S;
-        const uint32_t ph = (uint32_t)(kb / S) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
-          if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 1u; }
-          ok = false;
-          break;
-        }
-        mbar_expect_tx(full_bar(s), STAGE_BYTES);
-        const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
-        tma_load_2d(sa, &map_a, (kb0 + kb) * UM_BK, m0, full_bar(s));
-        tma_load_2d(sa + A_BYTES, &map_b0, (kb0 + kb) * UM_BK, row_b0, full_bar(s));
-        tma_load_2d(sa + A_BYTES + B_HALF_BYTES, &map_b1, (kb0 + kb) * UM_BK, row_b1, full_bar(s));
-        ++issued;
-      }
-      // Do not leave while copies may still be landing in this CTA's shared memory.
-      const int first = issued > S ? issued - S : 0;
-      for (int kb = first; kb < issued; ++kb) {
-        volatile uint32_t no_abort = 0;
-        mbar_wait(full_bar(kb % S), (uint32_t)(kb / S) & 1u, &no_abort);
-      }
-    }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(BN);
-      bool ok = true;
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % S;
-        const uint32_t ph = (uint32_t)(kb / S) & 1u;
-        if (!mbar_wait(full_bar(s), ph, abort_flag)) {
-          if (!*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 2u; }
-          ok = false;
-          break;
-        }
-        tc_fence_after();
-        const uint32_t sa = smem_u32(smem + (size_t)s * STAGE_BYTES);
-        const uint64_t da = make_smem_desc(sa);
-        const uint64_t db = make_smem_desc(sa + A_BYTES);
-#pragma unroll
-        for (int k = 0; k < UM_BK / 16; ++k) {
-          // advance 16 bf16 = 32 bytes = 2 descriptor units along K inside the swizzle row
-          tc_mma_f16(tmem_base, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
-        }
-        tc_commit(empty_bar(s));     // frees the stage once these MMAs have read it
-      }
-      if (ok) tc_commit(acc_bar);    // accumulator complete
-    }
-  } else {
-    // ---------------- epilogue (warps 2..5) ----------------
-    const int q = warp & 3;                        // TMEM lane quarter this warp may access
-    const int m = m0 + q * 32 + lane;
-    bool ok = mbar_wait(acc_bar, 0u, abort_flag);
-    if (!ok) *epi_fail = 1;
-    asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps agree on the outcome
-    ok = (*epi_fail == 0);
-    if (!ok) {
-      if (lane == 0 && !*abort_flag) { *abort_flag = 1; atomicExch(args.status, 1u); args.status[1] = 3u; }
-    } else if (splitk_epilogue<BN, Epi>(args, epi, tmem_base, q, lane, m, m0, tile, epi_last)) {
-      // handled by the split-K path
-    } else {
-      tc_fence_after();
-      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
-      if constexpr (Epi::kReduce) {
-        Top2 r = top2_empty();
-        const int col0 = tile * BN;
-#pragma unroll 1
-        for (int c = 0; c < BN; c += 16) {
-          float v[16];
-          tc_ld16(t_row + c, v);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int col = col0 + c + i;
-            if (epi.valid(col)) top2_push(r, v[i], col);
-          }
-        }
-        if (m < args.M) epi.part[(size_t)m * epi.n_tiles + tile] = r;
-      } else if constexpr (Epi::kDual) {
-        const int j0 = tile * HALF;
-#pragma unroll 1
-        for (int c = 0; c < HALF; c += 16) {
-          float a0[16], a1[16];
-          tc_ld16(t_row + c, a0);
-          tc_ld16(t_row + HALF + c, a1);
-          if (m < args.M && j0 + c < args.n_pairs) epi16(epi, m, j0 + c, a0, a1);
-        }
-      } else {
-        const int j0 = tile * BN;
-#pragma unroll 1
-        for (int c = 0; c < BN; c += 16) {
-          float a0[16];
-          tc_ld16(t_row + c, a0);
-          if (m < args.M && j0 + c < args.n_pairs) epi16(epi, m, j0 + c, a0, a0);
-        }
-      }
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 1) {
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)BN) : "memory");
-  }
-}
-
 // ---- host side ------------------------------------------------------------------------------------------------
 typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                     const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -518,20 +249,14 @@ struct UmmaState {
   int n_counters = 0;
   int target_ctas = 0;             // 0 = one CTA per SM
   int max_stages = UM_MAX_STAGES;
-  int allow_split = 1;
   int sm_smem = 233472;            // shared memory per SM
-  int skinny_ctas_per_sm = 2;      // co-resident CTAs a weight-streaming (M <= 128) launch aims for
-  int skinny_min_stages = 3;       // ... provided each still gets this many pipeline stages
-  int skinny_bn = 128;             // tile width of plain epilogues in that regime
   int pdl = 1;                     // launch with the programmatic-serialisation attribute
   int stream_cluster = 1;          // persistent kernel: K slices of a tile on one thread block cluster, reduced through DSMEM
   int max_clusters[9] = {0, 148, 74, 45, 33, 26, 22, 15, 15};   // [c]: clusters of c one-per-SM CTAs that can be resident at once (queried at init)
   int stream_half_sm = 1;          // persistent kernel: cap shared memory at half an SM when three stages still fit
-  int use_stream = 1;              // M <= 128: use the persistent weight-streaming kernel (gemm_stream.cuh)
   int stream_issuers = 1;          // MMA-issuing warps with one row tile per CTA (two row tiles always use two); measured: no gain from 2
-  int stream_two_tiles = 1;        // ... also for 129..256 rows: 1 = two row tiles per CTA, 2 = two row groups, 0 = no
-  int stream_big_mt = 3;           // ... and for more rows: 1 or 2 row tiles per CTA, 3 = whichever fills the SMs better,
-                                   // 0 = leave those to the tiled kernel
+  int stream_two_tiles = 1;        // 129..256 rows: 1 = two row tiles per CTA, 2 = two row groups
+  int stream_big_mt = 3;           // ... and for more rows: 1 or 2 row tiles per CTA, 3 = whichever fills the SMs better
   int stream_bn = 0;               // its tile width with one row tile (0 = automatic)
   int stream_bn2 = 0;              // ... and with two row tiles
   int stream_bn_dual = 0;          // tile width of dual epilogues: 0 = automatic, 192 or 256
@@ -583,54 +308,6 @@ inline const CUtensorMap* umma_map(UmmaState& st, const void* base, int rows, in
 constexpr int UM_HEAD_BN = 256;
 inline int umma_head_tiles(int vocab) { return (vocab + UM_HEAD_BN - 1) / UM_HEAD_BN; }
 
-// Launch shape of one GEMM, chosen by umma_gemm.
-struct UmmaPlan {
-  int splits = 1;        // split-K factor
-  int a_rows = UM_BM;    // rows of the activation box
-  int smem_cap = 0;      // dynamic shared memory the CTA may use (0 = the device maximum): a lower cap lets two CTAs share an SM
-};
-
-template <int BN, typename Epi>
-int umma_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
-                int n_rows_w, const Epi& epi, unsigned* status, UmmaPlan plan) {
-  const int stage = plan.a_rows * UM_BK * 2 + BN * UM_BK * 2;
-  // the MMA always reads 128 activation rows from the stage: rows past the box come from the rest of the stage (or, for
-  // narrow tiles, from the padding appended here) and only feed accumulator rows that are never stored
-  const int pad = stage < UM_BM * UM_BK * 2 ? UM_BM * UM_BK * 2 - stage : 0;
-  const int aux = 1024 /*alignment slack*/ + 8 * (2 * UM_MAX_STAGES + 1) + 16 + pad;
-  const int cap = plan.smem_cap > 0 && plan.smem_cap < st.max_smem ? plan.smem_cap : st.max_smem;
-  int stages = (cap - aux) / stage;
-  if (stages > st.max_stages) stages = st.max_stages;
-  int splits = plan.splits;
-  const int num_kb = K / UM_BK;
-  const int kb_per_split = (num_kb + splits - 1) / splits;
-  splits = (num_kb + kb_per_split - 1) / kb_per_split;      // no empty split
-  if (stages > kb_per_split) stages = kb_per_split;
-  if (stages < 1) { st.err = "not enough shared memory"; return -2; }
-  const size_t smem = (size_t)stages * stage + aux;
-  static bool attr_set = false;   // per instantiation
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(k_gemm_umma<BN, Epi>, cudaFuncAttributeMaxDynamicSharedMemorySize, st.max_smem);
-    if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -3; }
-    attr_set = true;
-  }
-  if (st.cache.size() > 4096) st.cache.clear();
-  const CUtensorMap* ma = umma_map(st, A, M, K, plan.a_rows);
-  const CUtensorMap* mb0 = umma_map(st, W0, n_rows_w, K, BN / 2);
-  const CUtensorMap* mb1 = umma_map(st, W1, n_rows_w, K, BN / 2);
-  if (!ma || !mb0 || !mb1) return -4;
-  const int per_tile = Epi::kDual ? BN / 2 : BN;
-  const int m_fast = Epi::kReduce ? 1 : 0;
-  dim3 grid((NP + per_tile - 1) / per_tile, (M + UM_BM - 1) / UM_BM);
-  if (m_fast) grid = dim3(grid.y, grid.x);
-  grid.z = splits;
-  UmmaArgs args{M, NP, K, num_kb, stages, plan.a_rows, m_fast, splits, kb_per_split, st.scratch, st.counters, status};
-  cudaError_t e = launch_k(st.pdl, k_gemm_umma<BN, Epi>, grid, dim3(UM_THREADS), smem, stream, *ma, *mb0, *mb1, args, epi);
-  if (e == cudaSuccess) e = cudaGetLastError();
-  if (e != cudaSuccess) { st.err = cudaGetErrorString(e); return -5; }
-  return 0;
-}
-
 template <typename Epi> int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn);
 template <int BN, int MT, int NI, typename Epi>
 int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
@@ -663,26 +340,14 @@ int stream_dispatch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf1
   return -7;
 }
 
-// Tile-width and split-K choice.
-//  * Problems with at most 256 activation rows go to the persistent weight-streaming kernel (gemm_stream.cuh) when it
-//    can take them; the rules below cover the rest.
-//  * Large problems (at least one CTA per SM without splitting) take the widest tile, one CTA per SM, deepest pipeline.
-//  * Single-row-tile problems (M <= 128) are bound by streaming the weights from HBM once.  Measured on B200, one
-//    CTA per SM that fetches 128 bytes per weight row per stage tops out near 3.7 TB/s however deep its pipeline is,
-//    while two co-resident CTAs per SM (or 256 bytes per row per stage) reach 5.3 TB/s.  So these launches load only
-//    the activation rows that exist (a box of 8..128 rows), cap their shared memory at half an SM so that two CTAs
-//    fit, and split K until both CTA slots of every SM are filled in a single wave.
-//  * The rotary epilogue needs both partners of a pair inside one head, which caps its tile at head_dim columns.
+// Tile-width choice for the persistent kernel (the K split follows from the tile count, see stream_launch).
+//  * The rotary epilogue needs both partners of a pair inside one head: its half tiles are fetched head by head.
+//  * A shape the kernel cannot take (none of a transformer layer's: it would need more than 4096 column tiles in a
+//    launch whose tiles are split between CTAs) is an error, not a fallback.
 template <typename Epi>
 int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
               int n_rows_w, const Epi& epi, unsigned* status) {
   if (K % UM_BK) { st.err = "K must be a multiple of 64"; return -6; }
-  const int mt = (M + UM_BM - 1) / UM_BM;
-  UmmaPlan plan;
-  if (mt == 1) {
-    plan.a_rows = 8;
-    while (plan.a_rows < M) plan.a_rows *= 2;
-  }
   if constexpr (Epi::kReduce) {
     {
       const int smt = stream_row_tiles<Epi>(st, M, NP, K, UM_HEAD_BN);
@@ -690,17 +355,10 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
         return stream_dispatch<Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 0, UM_HEAD_BN, smt,
                                     st.stream_issuers);
     }
-    if (mt == 1 && st.skinny_ctas_per_sm > 1) {
-      const int stage = plan.a_rows * UM_BK * 2 + UM_HEAD_BN * UM_BK * 2;
-      const int cap = (st.sm_smem / 2 - 1024) & ~1023;       // 2 x 256 accumulator columns fill the tensor memory
-      if ((cap - 2048) / stage >= st.skinny_min_stages) plan.smem_cap = cap;
-    }
-    return umma_launch<UM_HEAD_BN, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
+    st.err = "the tcgen05 head GEMM cannot take this shape";
+    return -8;
   } else {
     const int cols = Epi::kDual ? 2 * NP : NP;
-    const int num_kb = K / UM_BK;
-    int max_bn = 256;
-    if constexpr (std::is_same<Epi, EpiQKVRope<bf16>>::value) max_bn = 2 * epi.half;
     {
       // Tile width, from measurements on the LLaDA layer shapes at 2..256 rows: dual epilogues take 256 columns (128
       // pairs); plain ones take 128, which needs no K split with 96 tiles, except that a wide GEMM with at most 32
@@ -739,37 +397,8 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
         return stream_dispatch<Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, box_rows, sbn, smt,
                                     st.stream_issuers);
     }
-    int bn = max_bn;
-    const long big_tiles = (long)mt * ((cols + max_bn - 1) / max_bn);
-    if (big_tiles < st.n_sm) {
-      bn = Epi::kDual ? max_bn : (max_bn < st.skinny_bn ? max_bn : st.skinny_bn);
-      const long tiles = (long)mt * ((cols + bn - 1) / bn);
-      int slots = st.n_sm;
-      if (mt == 1 && st.skinny_ctas_per_sm > 1) {
-        const int stage = plan.a_rows * UM_BK * 2 + bn * UM_BK * 2;
-        const int cap = (st.sm_smem / st.skinny_ctas_per_sm - 1024) & ~1023;
-        if ((cap - 2048) / stage >= st.skinny_min_stages) {
-          plan.smem_cap = cap;
-          slots = st.n_sm * st.skinny_ctas_per_sm;
-        }
-      }
-      if (st.target_ctas > 0) slots = st.target_ctas;
-      if (st.allow_split && st.scratch != nullptr && tiles < slots) {
-        int splits = (int)(slots / tiles);
-        if (splits > num_kb / 4) splits = num_kb / 4;
-        if (splits < 1) splits = 1;
-        while (splits > 1 && ((size_t)tiles * splits * UM_BM * bn * sizeof(float) > st.scratch_bytes ||
-                              tiles > st.n_counters))
-          --splits;
-        plan.splits = splits;
-      }
-    }
-    switch (bn) {
-      case 256: return umma_launch<256, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
-      case 128: return umma_launch<128, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
-      case 64: return umma_launch<64, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
-      default: return umma_launch<32, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, plan);
-    }
+    st.err = "the tcgen05 GEMM cannot take this shape";
+    return -8;
   }
 }
 

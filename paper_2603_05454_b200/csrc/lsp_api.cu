@@ -781,25 +781,20 @@ int lsp_debug_set(lsp_ctx* c, int key, int value) {
 #ifndef LSP_NO_UMMA
   else if (key == 10) c->umma.target_ctas = value;
   else if (key == 11) c->umma.max_stages = value < 1 ? 1 : (value > UM_MAX_STAGES ? UM_MAX_STAGES : value);
-  else if (key == 12) c->umma.allow_split = value;
   else if (key == 25) { c->pdl = value ? 1 : 0; c->umma.pdl = c->pdl; }
-  else if (key == 16) c->umma.use_stream = value;
   else if (key == 17) c->umma.stream_grid_mode = value;
   else if (key == 18) c->umma.stream_even_max_rows = value;
-  else if (key == 19) c->umma.stream_two_tiles = value;
+  else if (key == 19) c->umma.stream_two_tiles = value == 2 ? 2 : 1;
   else if (key == 27) c->umma.stream_half_sm = value ? 1 : 0;
   else if (key == 29) c->umma.stream_cluster = value ? 1 : 0;
   else if (key == 32) c->umma.stream_bn_dual = (value == 192 || value == 256) ? value : 0;
   else if (key == 33) c->umma.stream_exchange = value ? 1 : 0;
   else if (key == 26) c->umma.stream_issuers = value == 1 ? 1 : 2;
-  else if (key == 24) c->umma.stream_big_mt = (value >= 1 && value <= 3) ? value : 0;
-  else if (key == 20) c->umma.stream_bn2 = (value == 256 || value == 128 || value == 64) ? value : 0;
-  else if (key == 23) c->umma.stream_bn = (value == 256 || value == 128 || value == 64) ? value : 0;
+  else if (key == 24) c->umma.stream_big_mt = (value == 1 || value == 2) ? value : 3;
+  else if (key == 20) c->umma.stream_bn2 = (value == 256 || value == 128) ? value : 0;
+  else if (key == 23) c->umma.stream_bn = (value == 256 || value == 128) ? value : 0;
   else if (key == 21) c->umma.stream_atoms = value;
   else if (key == 22) c->umma.stream_min_stages2 = value < 2 ? 2 : value;
-  else if (key == 13) c->umma.skinny_ctas_per_sm = value < 1 ? 1 : value;
-  else if (key == 14) c->umma.skinny_min_stages = value < 1 ? 1 : value;
-  else if (key == 15) c->umma.skinny_bn = (value == 64 || value == 32) ? value : 128;
 #endif
   else return fail(c, LSP_ERR_ARG, "lsp_debug_set: unknown key %d", key);
   return LSP_OK;

@@ -19,19 +19,15 @@ extern "C" {
  *   4  lsp_op_linear enqueues the operation this many times
  *   5  repetition r reads its weights at W + (r mod value) * N * K elements, so a buffer of several weight copies keeps
  *      the L2 cold
- * tcgen05 GEMM:
- *   10 CTAs a small-M GEMM is split into (0 = one per SM)          11 maximum pipeline stages
- *   12 allow split-K (1) or not (0)
- *   13 CTAs per SM a weight-streaming launch of the tiled kernel aims for
- *   14 fewest pipeline stages it accepts for that                   15 its tile width for plain epilogues (32, 64, 128)
- *   16 GEMMs use the persistent weight-streaming kernel (1, default) or the tiled one (0)
+ * tcgen05 GEMM (the persistent kernel k_gemm_stream):
+ *   10 CTAs a launch whose tiles are split is dealt to (0 = by the tile count)          11 maximum pipeline stages
  *   17 grid of the persistent kernel (0 by row count, 1 one CTA per SM with even shares, 2 a multiple of the tile count)
  *   18 row count up to which mode 0 takes even shares
- *   19 the persistent kernel also takes 129..256 rows: 1 = two row tiles per CTA (default), 2 = two row groups, 0 = no
- *   20 its tile width for those (0 = automatic, 64, 128, 256)
+ *   19 129..256 rows: 1 = two row tiles per CTA (default), 2 = two row groups
+ *   20 its tile width for those (0 = automatic, 128, 256)
  *   21 64-element K atoms per pipeline stage (0 = automatic, 1, 2)   22 fewest two-atom stages the automatic choice accepts
- *   23 its tile width for up to 128 rows (0 = automatic, 64, 128, 256)
- *   24 row tiles per CTA above 256 rows (1, 2, 3 = automatic, default; 0 = the tiled kernel takes those)
+ *   23 its tile width for up to 128 rows (0 = automatic, 128, 256)
+ *   24 row tiles per CTA above 256 rows (1, 2, 3 = automatic, default)
  *   25 launch the step's kernels with programmatic dependent launch (1, default) or plainly (0)
  *   26 MMA-issuing warps of the persistent kernel with one row tile per CTA (1, default, or 2)
  *   27 the persistent kernel caps its shared memory at half an SM when three stages still fit (1, default)
