@@ -404,7 +404,7 @@ def run_decode_bench(wl, dev, rank, world, peaks, steps, warmup, sampler=None, w
         res["d2h"] = host_out.numel() * 4
         assert int((host_out == sh.mask_id).sum()) == 0 and bool((host_out[:, :P] == host_in[:, :P]).all())
 
-    # Section 8(f)4-style variants of the loop on the same resident decoder: block lengths kept on the device (the host
+    # Variants of the loop on the same resident decoder: block lengths kept on the device (the host
     # enqueues pass k+1 before it has read L_k) and the in-place K/V layout (the append degenerates to a length bump).
     # The synchronous loop with the staged layout and the append copy (timed above) stays the contract.
     if variants:

@@ -21,7 +21,7 @@ The yardstick is E = oracle_bf16 - exact.  The CUDA path is held to it:
     as close to exact arithmetic as the oracle's own bf16 model does;
   * every pass:  max|gpu - oracle_bf16| <= 3 max|E| (two independent roundings of the same quantity);
   * an argmax may differ from the oracle's only where the oracle's own margin delta is below 2 max|E_delta|.
-The measured figures are printed (pytest -s), written to $LSP_PARITY_REPORT when set, and tabulated in the design doc.
+The measured figures are printed (pytest -s) and written to $LSP_PARITY_REPORT when set.
 """
 import importlib.util
 import os
