@@ -263,6 +263,9 @@ struct UmmaState {
   int stream_exchange = 1;         // clusters of 2 exchange half tiles instead of publishing whole partial tiles
   int stream_atoms = 0;            // K atoms per stage: 0 = two when stream_min_stages2 such stages fit, else 1 or 2 as given
   int stream_min_stages2 = 3;
+  int swap_min_rows = 129;         // row counts [min, max] that take the operand-swapped kernel (gemm_swap.cuh); max 0 = never
+  int swap_max_rows = 256;
+  int swap_force = 0;              // 1: take it whenever it can run (tests), not only where it was measured to pay
   int stream_grid_mode = 2;        // its grid: 0 = by row count, 1 = one CTA per SM (even shares), 2 = multiple of the tile count
   int stream_even_max_rows = 0;    // mode 0: even shares up to this many activation rows
   std::string err;
@@ -309,6 +312,9 @@ constexpr int UM_HEAD_BN = 256;
 inline int umma_head_tiles(int vocab) { return (vocab + UM_HEAD_BN - 1) / UM_HEAD_BN; }
 
 template <typename Epi> int stream_row_tiles(const UmmaState& st, int M, int NP, int K, int bn);
+template <int NACC, typename Epi>
+int swap_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
+                int n_rows_w, const Epi& epi, unsigned* status, int box_rows);
 template <int BN, int MT, int NI, typename Epi>
 int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0, const bf16* W1, int M, int NP, int K,
                   int n_rows_w, const Epi& epi, unsigned* status, int box_rows);
@@ -359,6 +365,15 @@ int umma_gemm(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16* W0,
     return -8;
   } else {
     const int cols = Epi::kDual ? 2 * NP : NP;
+    if (M >= st.swap_min_rows && M <= st.swap_max_rows) {
+      // 129..256 rows: the tensor pipe bounds the launch, and with the operands swapped its time follows the row count
+      int rc;
+      if constexpr (std::is_same<Epi, EpiQKVRope<bf16>>::value) rc = swap_launch<2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, epi.half);
+      else if constexpr (Epi::kDual) rc = st.swap_force ? swap_launch<2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 0) : 1;   // gate/up: one K slice only, 96 CTAs of 3 MB intake each: the 192-wide row-major tiles win (measured)
+      else if (cols >= 8192) rc = swap_launch<2, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 0);
+      else rc = swap_launch<1, Epi>(st, stream, A, W0, W1, M, NP, K, n_rows_w, epi, status, 0);
+      if (rc <= 0) return rc;          // 1 = not a problem that kernel takes
+    }
     {
       // Tile width, from measurements on the LLaDA layer shapes at 2..256 rows: dual epilogues take 256 columns (128
       // pairs); plain ones take 128, which needs no K split with 96 tiles, except that a wide GEMM with at most 32

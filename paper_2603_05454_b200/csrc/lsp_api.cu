@@ -20,6 +20,7 @@
 #include "misc_kernels.cuh"
 #ifndef LSP_NO_UMMA
 #include "gemm_stream.cuh"
+#include "gemm_swap.cuh"
 #include "attention_umma.cuh"
 #endif
 
@@ -774,6 +775,9 @@ int lsp_debug_set(lsp_ctx* c, int key, int value) {
   if (!c) return LSP_ERR_ARG;
   if (key == 28) c->attn_umma_min_rows = value;
   else if (key == 31) c->lag_tail = value < 1 ? 1 : value;
+  else if (key == 36) c->umma.swap_min_rows = value;
+  else if (key == 37) c->umma.swap_max_rows = value;
+  else if (key == 38) c->umma.swap_force = value ? 1 : 0;
   else if (key == 30) c->attn_cluster = value ? 1 : 0;
   else if (key == 3) c->async_ops = value;
   else if (key == 4) c->op_repeat = value < 1 ? 1 : value;

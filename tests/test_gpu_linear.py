@@ -225,3 +225,41 @@ def test_linear_bf16_third_model_shape(M):
         np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * (2 if op == 2 else 1),
                                    atol=rtol * np.abs(ref).max() * 0.05, err_msg=f"M={M} N={N} K={K} op={op}")
     dec.close()
+
+
+@pytest.mark.parametrize("M", [1, 16, 17, 100, 129, 144, 177, 200, 256])
+def test_linear_bf16_operand_swapped_kernel(M):
+    """The operand-swapped kernel (weights as the 128-row MMA operand, activation rows as N in steps of 16), forced on for
+    every row count up to 256: one and two accumulators, K slices on clusters of 1, 2 and 4, ragged last tiles, all three
+    epilogues, twice (bit-identical: the K slices are summed in rank order)."""
+    dec = _dec("bf16")
+    dec.debug_set(36, 1)
+    dec.debug_set(37, 256)
+    dec.debug_set(38, 1)
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    rtol = 1.0 / 128
+    for (N, K) in ((4096, 4096), (12288, 4096), (1152, 512), (384, 256), (3584, 18944), (4608, 3584), (144, 192)):
+        A = S.normal((M, K), 7, 1, 1.0, torch.bfloat16, DEV)
+        W = S.normal((N, K), 7, 2, 0.03, torch.bfloat16, DEV)
+        W2 = S.normal((N, K), 7, 3, 0.03, torch.bfloat16, DEV)
+        X0 = S.normal((M, N), 7, 4, 1.0, torch.bfloat16, DEV)
+        a, w, w2, x0 = f64(A), f64(W), f64(W2), f64(X0)
+        tag = f"M={M} N={N} K={K}"
+        out = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+        outs = []
+        for _ in range(2):
+            out.fill_(float("nan"))
+            dec.op_linear(0, A, W, None, out)
+            ref = a @ w.T
+            np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05, err_msg=tag)
+            outs.append(out.clone())
+        assert torch.equal(outs[0], outs[1]), tag
+        xr = X0.clone()
+        dec.op_linear(1, A, W, None, xr)
+        ref = x0 + a @ w.T
+        np.testing.assert_allclose(f64(xr), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05, err_msg=tag)
+        dec.op_linear(2, A, W, W2, out)
+        g, u = a @ w.T, a @ w2.T
+        ref = g / (1 + np.exp(-g)) * u
+        np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05, err_msg=tag)
+    dec.close()
