@@ -14,7 +14,7 @@ NEAR = oscan.FLAG_NEAR_THRESHOLD | oscan.FLAG_NEAR_TIE
 
 
 def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, max_steps=None, gains_seed=None,
-                    max_batch=1, extra_len=0, poison=False, inplace=False):
+                    max_batch=1, extra_len=0, poison=False, inplace=False, debug=None):
     """Runs the GPU path step by step, committing the ORACLE's lengths, and compares every step's outputs."""
     from paper_2603_05454_b200 import LSPDecoder
     tol = tol_for(shape.dtype)
@@ -50,6 +50,8 @@ def _teacher_forced(shape, seed, P, G, sched, delim, impl=None, attn_impl=None, 
         dec.workspace[-((stage + 255) // 256 * 256):].view(it).fill_(pat)
     if inplace:
         dec.set_option(3, 1)
+    for k, v in (debug or {}).items():
+        dec.debug_set(k, v)
     if impl is not None:
         dec.set_option(0, impl)
     if attn_impl is not None:
@@ -346,3 +348,16 @@ def test_in_place_kv_layout_free_running_batch_equals_the_staged_layout_where_un
         if same:
             assert np.array_equal(out[0][0][b, :Ps[b] + Gs[b]], out[1][0][b, :Ps[b] + Gs[b]])
         assert (out[1][0][b, :Ps[b] + Gs[b]] != sh.mask_id).all()
+
+
+@pytest.mark.parametrize("inplace", [False, True])
+def test_operand_swapped_gemms_in_a_whole_decode(inplace):
+    """Every layer GEMM of a decode through the operand-swapped kernel (forced on at every row count it can run at): the
+    rotary epilogue with its K/V staging (or the in-place layout's cache slots), the residual updates and the SwiGLU
+    pair, with grouped-query heads, against the oracle step by step."""
+    from paper_2603_05454_b200 import SchedCfg
+    sh = S.ModelShape(2, 512, 4, 2, 128, 1024, 4096, dtype="bf16", head_scale=1.5, w_std=0.044)
+    _teacher_forced(sh, 71, 150, 170, SchedCfg(mode=2, fixed_k=45), (1, 200), max_steps=5, inplace=inplace,
+                    debug={36: 1, 38: 1})
+    _teacher_forced(sh, 72, 20, 60, SchedCfg(tau=0.04), (1, 400), inplace=inplace, debug={36: 1, 38: 1}, poison=True,
+                    max_batch=2, extra_len=30)

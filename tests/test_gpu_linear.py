@@ -137,11 +137,12 @@ def test_linear_bf16_cluster_split_of_two_row_tiles(case):
 
 def test_linear_bf16_seeded_random_shapes_and_kernel_options():
     """Sixty seeded random (rows, columns, K, option) combinations across the row regimes (one tile, two tiles, row
-    groups), the split paths (clusters of 2..8, half-tile exchange, rounds, global scratch) and the tile widths."""
+    groups), the split paths (clusters of 2..8, half-tile exchange, rounds, global scratch), the tile widths, and the
+    operand-swapped kernel forced on."""
     import random
     rng = random.Random(7)
     dec = _dec("bf16")
-    defaults = {29: 1, 33: 1, 20: 0, 23: 0, 32: 0, 17: 2, 24: 3}
+    defaults = {29: 1, 33: 1, 20: 0, 23: 0, 32: 0, 17: 2, 24: 3, 36: 129, 38: 0}
     f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
     rows = [1, 2, 5, 17, 32, 33, 64, 100, 128, 129, 190, 256, 257, 300, 400, 512, 640, 768, 1000, 1100, 1536, 2100]
     done = 0
@@ -152,9 +153,11 @@ def test_linear_bf16_seeded_random_shapes_and_kernel_options():
             continue
         opts = {}
         for key, p, vals in ((29, 0.2, [0]), (33, 0.2, [0]), (20, 0.15, [128, 256]), (23, 0.15, [128, 256]),
-                             (32, 0.15, [192, 256]), (17, 0.1, [1]), (24, 0.1, [1, 2])):
+                             (32, 0.15, [192, 256]), (17, 0.1, [1]), (24, 0.1, [1, 2]), (38, 0.3, [1])):
             if rng.random() < p:
                 opts[key] = rng.choice(vals)
+        if opts.get(38):
+            opts[36] = 1                    # the operand-swapped kernel at every row count up to 256, on any shape it can run
         for k, v in {**defaults, **opts}.items():
             dec.debug_set(k, v)
         A = S.normal((M, K), done, 1, 1.0, torch.bfloat16, DEV)
