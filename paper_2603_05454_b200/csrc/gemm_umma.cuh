@@ -2,7 +2,7 @@
 //
 //   acc[m, c] = sum_k A[m, k] * Wt[c, k]        A: [M, K] bf16 row-major, Wt: weight rows, K-major, fp32 accumulate
 //
-// This header holds the PTX wrappers (mbarrier with bounded waits, TMA tile loads without multicast, tcgen05.mma /
+// This header holds the PTX wrappers (mbarrier with bounded waits, TMA tile loads (every CTA fetches its own tiles), tcgen05.mma /
 // .commit / .ld), the shared-memory and instruction descriptors, the vectorised fused epilogues (store / residual /
 // SwiGLU / rotary + K/V staging), the host state (tensor-map cache, tuning fields) and the dispatch that picks tile
 // width and row tiles per CTA.  The kernel itself is the persistent k_gemm_stream of gemm_stream.cuh; the attention
