@@ -48,6 +48,8 @@ struct StreamArgs {
   int atoms;        // 64-element K atoms per stage (1 or 2)
   int box_rows;     // weight rows per TMA box: BN/2, or fewer when the rows of a half tile are not contiguous (rotary pairs)
   int stages;
+  int half_tile1;   // two row tiles, every CTA one whole tile, at most 192 rows: the second row tile's MMAs span 64
+                    // accumulator rows instead of 128 (its rows sit in the lower half of every warp's tensor-memory lanes)
   float* scratch;   // [gridDim.x][2][128 MT][BN] fp32 partial tiles
   unsigned* counters;  // one per column tile, zero between launches
   unsigned* status;
@@ -244,7 +246,7 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     // ---------------- MMA issuers ----------------
     const int is = warp == 1 ? 0 : 1;                   // issuer index
     if (lane == 0 && is < NI) {
-      constexpr uint32_t idesc = make_idesc(BN);
+      const uint32_t idesc = (MT == 2 && is == 1 && args.half_tile1) ? make_idesc_m64(BN) : make_idesc(BN);
       int seg = 0;
       bool ok = true;
       int s = 0;
@@ -317,7 +319,8 @@ k_gemm_stream(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
         // the accumulator is complete in tensor memory: each thread owns one row of every row tile
 #pragma unroll 1
         for (int mt = 0; mt < MT; ++mt) {
-          const int m = row0 + mt * UM_BM + r_in;
+          int m = row0 + mt * UM_BM + r_in;
+          if (MT == 2 && mt == 1 && args.half_tile1) m = lane < 16 ? row0 + UM_BM + q * 16 + lane : 0x7fffffff;   // 64-row accumulator
           Top2 red = top2_empty();
           // one chunk of 16 columns (or pairs) at a time; the next chunk's tensor-memory loads are in flight while this
           // one is converted and stored (with K-parity accumulators the extra loads are not pipelined)
@@ -774,8 +777,11 @@ int stream_launch(UmmaState& st, cudaStream_t stream, const bf16* A, const bf16*
       if (splits == 2 && st.stream_exchange && !(MT == 1 && NI == 2) && 2 * area >= MT * tile_bytes) cl_rounds = 0;
     }
   }
-  StreamArgs args{M, NP, n_tiles, row_groups, whole, cluster, cl_rounds, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, st.scratch,
-                  st.counters, status};
+  // at most 192 rows on two row tiles, every CTA one unsplit tile: 64-row MMAs for the second row tile
+  const int half_tile1 = (MT == 2 && !Epi::kReduce && st.stream_half_tile1 && row_groups == 1 && M <= UM_BM + 64 && grid == (int)T &&
+                          cluster == 0) ? 1 : 0;
+  StreamArgs args{M, NP, n_tiles, row_groups, whole, cluster, cl_rounds, kc, sh.a_rows, sh.atoms, box_rows, sh.stages, half_tile1,
+                  st.scratch, st.counters, status};
   cudaError_t e = launch_k(st.pdl, k_gemm_stream<BN, MT, NI, Epi>, dim3(grid), dim3(ST_THREADS), smem, stream, cluster, *ma, *mb0,
                            *mb1, args, epi);
   if (e == cudaSuccess) e = cudaGetLastError();

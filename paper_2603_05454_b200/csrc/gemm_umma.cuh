@@ -149,6 +149,10 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   return d;
 }
 // Instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128, N = BN.
+// (M = 64 puts accumulator row r in tensor-memory lane 32 (r / 16) + r % 16: the lower half of every warp's lane quarter.)
+__host__ __device__ constexpr uint32_t make_idesc_m64(int bn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(64 >> 4) << 24);
+}
 __host__ __device__ constexpr uint32_t make_idesc(int bn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(UM_BM >> 4) << 24);
 }
@@ -263,6 +267,7 @@ struct UmmaState {
   int stream_exchange = 1;         // clusters of 2 exchange half tiles instead of publishing whole partial tiles
   int stream_atoms = 0;            // K atoms per stage: 0 = two when stream_min_stages2 such stages fit, else 1 or 2 as given
   int stream_min_stages2 = 3;
+  int stream_half_tile1 = 1;       // 129..192 rows on two row tiles, unsplit: 64-row MMAs for the second row tile
   int swap_min_rows = 129;         // row counts [min, max] that take the operand-swapped kernel (gemm_swap.cuh); max 0 = never
   int swap_max_rows = 256;
   int swap_force = 0;              // 1: take it whenever it can run (tests), not only where it was measured to pay

@@ -778,6 +778,7 @@ int lsp_debug_set(lsp_ctx* c, int key, int value) {
   else if (key == 36) c->umma.swap_min_rows = value;
   else if (key == 37) c->umma.swap_max_rows = value;
   else if (key == 38) c->umma.swap_force = value ? 1 : 0;
+  else if (key == 39) c->umma.stream_half_tile1 = value ? 1 : 0;
   else if (key == 30) c->attn_cluster = value ? 1 : 0;
   else if (key == 3) c->async_ops = value;
   else if (key == 4) c->op_repeat = value < 1 ? 1 : value;
@@ -1365,7 +1366,7 @@ int lsp_linear_static(const void* A, const void* W, void* out, int M, int N, int
     static_msg(err, err_len, "lsp_linear_static: clearing the counters failed (%s)", cudaGetErrorString(e));
     return LSP_ERR_CUDA;
   }
-  StreamArgs args{M, N, n_tiles, 1, 0, 0, 1, kc, a_rows, atoms, kStaticBN / 2, stages, partials, counters, status};
+  StreamArgs args{M, N, n_tiles, 1, 0, 0, 1, kc, a_rows, atoms, kStaticBN / 2, stages, 0, partials, counters, status};
   EpiStore<bf16> epi{(bf16*)out, N};
   k_gemm_stream<kStaticBN, 1, 2, EpiStore<bf16>><<<grid, ST_THREADS, smem, stream>>>(ma, mb, mb, args, epi);
   e = cudaGetLastError();

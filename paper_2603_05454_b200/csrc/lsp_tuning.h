@@ -38,6 +38,7 @@ extern "C" {
  * tcgen05 attention:
  *   28 fewest (query row x group head) rows of a (sequence, KV head) for which the tcgen05 kernel is used (default 0)
  *   30 it splits a row tile's keys over a thread block cluster when there are few CTAs (1, default)
+ *   39 with 129..192 rows on two row tiles and unsplit tiles, the second row tile's MMAs span 64 rows (1, default)
  *   36, 37 fewest and most activation rows of a GEMM that takes the operand-swapped kernel (defaults 129 and 256;
  *      37 = 0: never)        38 take it whenever it can run (1), not only where it was measured to pay (0, default)
  * decode loop:

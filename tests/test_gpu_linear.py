@@ -266,3 +266,37 @@ def test_linear_bf16_operand_swapped_kernel(M):
         ref = g / (1 + np.exp(-g)) * u
         np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05, err_msg=tag)
     dec.close()
+
+
+@pytest.mark.parametrize("case", [(130, 12288, 256, {}), (150, 12288, 320, {}), (192, 12288, 256, {}), (177, 9600, 192, {}),
+                                  (160, 12288, 256, {32: 256}), (193, 12288, 256, {}), (150, 12288, 256, {39: 0}),
+                                  (140, 12288, 512, {37: 0})])
+def test_linear_bf16_second_row_tile_of_64_rows(case):
+    """129..192 rows on two row tiles with unsplit tiles (the SwiGLU GEMM of a wide FFN): the second row tile runs 64-row
+    MMAs, whose accumulator rows sit in the lower half of every warp's tensor-memory lanes.  Also the neighbouring cases
+    that must not take that path (193 rows; the option off; plain epilogues with the operand-swapped kernel off)."""
+    M, N, K, opts = case
+    dec = _dec("bf16")
+    for k, v in opts.items():
+        dec.debug_set(k, v)
+    A = S.normal((M, K), 9, 1, 1.0, torch.bfloat16, DEV)
+    W = S.normal((N, K), 9, 2, 0.05, torch.bfloat16, DEV)
+    W2 = S.normal((N, K), 9, 3, 0.05, torch.bfloat16, DEV)
+    X0 = S.normal((M, N), 9, 4, 1.0, torch.bfloat16, DEV)
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    a, w, w2, x0 = f64(A), f64(W), f64(W2), f64(X0)
+    rtol = 1.0 / 128
+    out = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device=DEV)
+    dec.op_linear(2, A, W, W2, out)
+    g, u = a @ w.T, a @ w2.T
+    ref = g / (1 + np.exp(-g)) * u
+    np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol * 2, atol=rtol * np.abs(ref).max() * 0.05)
+    out.fill_(float("nan"))
+    dec.op_linear(0, A, W, None, out)
+    ref = a @ w.T
+    np.testing.assert_allclose(f64(out), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05)
+    xr = X0.clone()
+    dec.op_linear(1, A, W, None, xr)
+    ref = x0 + a @ w.T
+    np.testing.assert_allclose(f64(xr), dlm.round_bf16(ref), rtol=rtol, atol=rtol * np.abs(ref).max() * 0.05)
+    dec.close()
