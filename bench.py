@@ -56,9 +56,9 @@ CLASS_SOURCES = {
 }
 NCU_TRAFFIC = {
     # k_gemm_stream<128,1,1,EpiStore>, M 64, N 12288, K 4096: profiles/k_gemm_stream_M64_N12288_K4096.md
-    "gemm": {"captured_bytes": 104.82e6, "algorithmic_bytes": 102.8e6, "src": "0d1aa7edb1ac"},
+    "gemm": {"captured_bytes": 105.06e6, "algorithmic_bytes": 102.8e6, "src": "34127c2c8b24"},
     # k_gemm_stream<256,1,1,EpiHead>, 64 rows: profiles/k_gemm_stream_head_M64_V126464.md
-    "head": {"captured_bytes": 1063.4e6, "algorithmic_bytes": 1037.0e6, "src": "0d1aa7edb1ac"},
+    "head": {"captured_bytes": 1062.8e6, "algorithmic_bytes": 1037.0e6, "src": "34127c2c8b24"},
     # k_attn_umma, 16 x (128 query rows over 2048 keys): profiles/k_attn_umma_B16_F1920.md
     "attn": {"captured_bytes": 569.2e6, "algorithmic_bytes": 570.4e6, "src": "196044e4044b"},
     # k_commit_append of a 16 x 1920-row prompt block: profiles/k_commit_append_prompt_B16_P1920.md
