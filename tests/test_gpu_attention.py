@@ -13,11 +13,11 @@ from gpu_util import DEV
 pytestmark = pytest.mark.gpu
 
 # The kernel feeds bf16 softmax weights (relative error 2^-9 each) to the tensor core and rounds the output once; the
-# oracle keeps the weights in fp64.  With |v| <= 4.9 (the generator's support) and independent errors over the keys the
-# difference stays far below 2^-8 * max|v| = 1.9e-2: the bound asserted is the benchmark's 2e-2 absolute, and the
-# measured maximum is printed (pytest -s) and asserted against a tighter, measured ceiling.
+# oracle keeps the weights in fp64 and is rounded to bf16 here as well.  The two agree except where the last bit of the
+# bf16 output flips, so the difference is at most one bf16 ulp of the output: 7.8e-3 for |out| < 2 (the measured maximum
+# on B200, printed with pytest -s), 1.56e-2 for |out| < 4.  Asserted: the benchmark's 2e-2 absolute, and that ulp bound.
 ATOL = 2e-2
-MEASURED_CEILING = 8e-3
+MEASURED_CEILING = 1.6e-2
 
 
 def _run_case(hq, hkv, cache_len, rows, max_len, attn_impl=None, expect_cluster=None, seed=0, poison=False):
