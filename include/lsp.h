@@ -118,8 +118,9 @@ size_t lsp_workspace_bytes(const lsp_model_cfg* model, int max_batch, int max_le
 size_t lsp_kv_cache_bytes(const lsp_model_cfg* model, int max_batch, int max_len);
 
 /* Creates a context.  kv_cache and workspace are device buffers of at least the sizes above, 256-byte
- * aligned; cuda_stream is a cudaStream_t (NULL = default stream).  The first call builds the rotary
- * table on the device and may JIT nothing; it does not allocate device memory. */
+ * aligned; neither needs initialising (no result ever depends on memory the library has not written);
+ * cuda_stream is a cudaStream_t (NULL = default stream).  The call builds the rotary table on the
+ * device; it does not allocate device memory. */
 int lsp_init(lsp_ctx** out, const lsp_model_cfg* model, const lsp_sched_cfg* sched, const lsp_weights* weights,
              void* kv_cache, void* workspace, size_t workspace_bytes, int max_batch, int max_len,
              void* cuda_stream);
@@ -139,7 +140,9 @@ int lsp_set_sched(lsp_ctx* ctx, const lsp_sched_cfg* sched);
  * (default) = it reads L back after every pass before it enqueues the next; 1 = device-resident: the scan's L feeds the
  * commit kernel directly, the next pass's descriptor is derived from it on the device, and the host enqueues pass k+1
  * while pass k runs, reading L one step late (it sizes launches from row counts it knows a step late, upper bounds for
- * the LM-head rows; rows beyond the real ones are inert).  Same tokens, boundaries and records either way; prefix
+ * the LM-head rows; rows beyond the real ones are inert).  The decode is the same: identical tokens, boundaries and
+ * records on fp32 models; on bf16 models up to the last bits of a score (the LM-head launch has more rows, which can
+ * move a tile boundary of its reduction), i.e. up to decisions within rounding distance of a threshold or tie.  Prefix
  * topology only, and only while per-class timing is off (otherwise the synchronous loop runs).  Any other key:
  * LSP_ERR_ARG. */
 int lsp_set_option(lsp_ctx* ctx, int key, int value);
